@@ -1,0 +1,146 @@
+// CPU oracle for the signSGD / Signum / majority-vote step (Bernstein et al.,
+// "signSGD: Compressed Optimisation for Non-Convex Problems", Algorithms 1-3).
+//
+// TEST INFRASTRUCTURE ONLY.  This file is the slow, plain definition that the
+// CUDA library is checked against.  It shares no code, header, table or helper
+// with the CUDA sources, and the product never calls it: only the test-suite,
+// the smoke check and the benchmark's cpu-baseline leg load this library.
+//
+// Everything is written as scalar loops over *unpacked* values (one byte per
+// sign), with packing into words kept in a separate trivial loop, so that an
+// arithmetic mistake and a packing mistake show up in different tests.
+//
+// Conventions the paper leaves open and this oracle fixes (each is pinned by a
+// test against brute force or a closed form):
+//   * sign(v) is encoded in one bit as  bit = !(v < 0): zero, -0.0 and NaN all
+//     count as +1, so that "1-bit" (Sec. 1, Table 1) holds without a third symbol.
+//   * an even-M tie, sum_m sign(g_m) = 0 in Algorithm 3, resolves to +1;
+//     equivalently vote = [P >= ceil(M/2)] with P the number of +1 votes.
+//   * word j of a packed row holds elements 32j .. 32j+31, least significant
+//     bit first; bits at positions >= d are 0.
+//   * momentum (Algorithm 2, second step) is evaluated in fp32 as
+//         omb = fl(1 - beta);  t = fl(omb * g);  m <- fma(beta, m, t)
+//     i.e. two roundings per element, the last one a fused multiply-add.
+//   * each worker keeps its own momentum and sends sign(m_new)  (Algorithm 2
+//     run per worker, feeding Algorithm 3's server); beta = 0 gives Algorithm 3
+//     as printed.
+//
+// All pointers are HOST pointers.  Parity status: every function below is
+// pinned by tests that do not call back into this file (brute force in Python,
+// closed forms in extended precision, invariants, bitwise MAJ3).
+
+#include <cmath>
+#include <cstddef>
+#include <cstdint>
+#include <cstdlib>
+#include <vector>
+
+extern "C" {
+
+// Number of 32-bit words that hold d one-bit signs (Table 1: d bits per vector).
+size_t ssgd_words_ref(size_t d) { return d / 32 + (d % 32 != 0 ? 1 : 0); }
+
+// sign(.) of Algorithms 1-3 on one row, unpacked: s[i] = 1 for +1, 0 for -1.
+void ssgd_sign_unpacked_ref(const float* v, size_t d, uint8_t* s) {
+  for (size_t i = 0; i < d; ++i) {
+    s[i] = (v[i] < 0.0f) ? 0 : 1;
+  }
+}
+
+// The 1-bit wire format: LSB-first words, padding bits zero.
+void ssgd_pack_bits_ref(const uint8_t* s, size_t d, uint32_t* words) {
+  const size_t W = ssgd_words_ref(d);
+  for (size_t j = 0; j < W; ++j) words[j] = 0u;
+  for (size_t i = 0; i < d; ++i) {
+    if (s[i]) words[i / 32] |= (uint32_t(1) << (i % 32));
+  }
+}
+
+void ssgd_unpack_bits_ref(const uint32_t* words, size_t d, uint8_t* s) {
+  for (size_t i = 0; i < d; ++i) {
+    s[i] = uint8_t((words[i / 32] >> (i % 32)) & 1u);
+  }
+}
+
+// Algorithm 1 / Algorithm 3 worker side: every worker w sends sign(g_w).
+void ssgd_sign_pack_ref(const float* g, size_t M, size_t d, size_t ld,
+                        uint32_t* bits, size_t ldw) {
+  std::vector<uint8_t> s(d);
+  for (size_t w = 0; w < M; ++w) {
+    ssgd_sign_unpacked_ref(g + w * ld, d, s.data());
+    ssgd_pack_bits_ref(s.data(), d, bits + w * ldw);
+  }
+}
+
+// Algorithm 2, second step, on one row, in place: m <- beta m + (1-beta) g.
+void ssgd_momentum_ref(const float* g, float* m, size_t d, float beta) {
+  const float omb = 1.0f - beta;
+  for (size_t i = 0; i < d; ++i) {
+    const float t = omb * g[i];
+    m[i] = std::fmaf(beta, m[i], t);
+  }
+}
+
+// Algorithm 2 per worker, then the sign of the *new* momentum is what is sent.
+void ssgd_signum_momentum_pack_ref(const float* g, float* m, size_t M, size_t d,
+                                   size_t ld, float beta, uint32_t* bits,
+                                   size_t ldw) {
+  std::vector<uint8_t> s(d);
+  for (size_t w = 0; w < M; ++w) {
+    ssgd_momentum_ref(g + w * ld, m + w * ld, d, beta);
+    ssgd_sign_unpacked_ref(m + w * ld, d, s.data());
+    ssgd_pack_bits_ref(s.data(), d, bits + w * ldw);
+  }
+}
+
+// Algorithm 3 server side on unpacked signs: count the +1 votes per element.
+void ssgd_vote_counts_ref(const uint32_t* bits, size_t M, size_t d, size_t ldw,
+                          int32_t* P) {
+  std::vector<uint8_t> s(d);
+  for (size_t i = 0; i < d; ++i) P[i] = 0;
+  for (size_t w = 0; w < M; ++w) {
+    ssgd_unpack_bits_ref(bits + w * ldw, d, s.data());
+    for (size_t i = 0; i < d; ++i) P[i] += s[i];
+  }
+}
+
+// Algorithm 3 server side: sign[ sum_m sign(g_m) ].  With P positive votes the
+// sum is P - (M - P) = 2P - M; it is >= 0 (tie counts as +1) iff 2P >= M.
+void ssgd_majority_vote_ref(const uint32_t* bits, size_t M, size_t d,
+                            size_t ldw, uint32_t* vote) {
+  std::vector<int32_t> P(d);
+  std::vector<uint8_t> s(d);
+  ssgd_vote_counts_ref(bits, M, d, ldw, P.data());
+  for (size_t i = 0; i < d; ++i) {
+    const long long sum = 2LL * P[i] - (long long)M;
+    s[i] = (sum < 0) ? 0 : 1;
+  }
+  ssgd_pack_bits_ref(s.data(), d, vote);
+}
+
+// Algorithm 3 worker side (also the last line of Algorithms 1 and 2):
+// x <- x - delta * sign(vote).
+void ssgd_sign_apply_ref(float* x, const uint32_t* vote, size_t d, float delta) {
+  std::vector<uint8_t> s(d);
+  ssgd_unpack_bits_ref(vote, d, s.data());
+  for (size_t i = 0; i < d; ++i) {
+    if (s[i]) x[i] = x[i] - delta;
+    else      x[i] = x[i] + delta;
+  }
+}
+
+// One whole step of Algorithm 3 with Signum workers.  beta == 0 is Algorithm 3
+// as printed (workers send sign(g)); m may then be NULL.
+void ssgd_signsgd_step_ref(float* x, const float* g, float* m, size_t M,
+                           size_t d, size_t ld, float beta, float delta,
+                           uint32_t* bits, size_t ldw, uint32_t* vote) {
+  if (beta == 0.0f && m == nullptr) {
+    ssgd_sign_pack_ref(g, M, d, ld, bits, ldw);
+  } else {
+    ssgd_signum_momentum_pack_ref(g, m, M, d, ld, beta, bits, ldw);
+  }
+  ssgd_majority_vote_ref(bits, M, d, ldw, vote);
+  ssgd_sign_apply_ref(x, vote, d, delta);
+}
+
+}  // extern "C"
