@@ -1,0 +1,136 @@
+/* signsgd.h -- C ABI of the B200 (sm_100a) signSGD / Signum / majority-vote library.
+ *
+ * The calls follow Algorithms 1-3 of Bernstein, Wang, Azizzadenesheli and
+ * Anandkumar, "signSGD: Compressed Optimisation for Non-Convex Problems":
+ * each of M workers turns its gradient (Algorithm 1) or its momentum
+ * (Algorithm 2) into one sign bit per parameter, a server takes the majority
+ * of the M bits per parameter, and every worker moves each parameter by
+ * -delta or +delta according to the voted bit (Algorithm 3).  Here the M
+ * workers are M rows of one buffer on one GPU.
+ *
+ * Notation: d parameters, M workers, W = ssgd_words(d) = ceil(d/32) words.
+ *
+ * Data layout (all fixed by this library; the paper only says "1-bit"):
+ *   g, m   float [M][ld]   row w at g + w*ld; elements d..ld-1 of a row are
+ *                          padding: they may be read, they are never written.
+ *   x      float [d]
+ *   bits   uint32 [M][ldw] row w at bits + w*ldw; word j of a row holds
+ *                          elements 32j..32j+31, least significant bit first;
+ *                          bit = 1 encodes sign +1, bit = 0 encodes sign -1;
+ *                          bits at positions >= d are written as 0; words
+ *                          W..ldw-1 of a row may be read, never written.
+ *   vote   uint32 [W]      same bit layout as one row of bits.
+ *
+ * Sign and tie rules: sign(v) -> bit !(v < 0), so +0, -0 and NaN encode +1;
+ * a vote with as many -1 as +1 (even M) resolves to +1, i.e. the voted bit is
+ * [P >= ceil(M/2)] with P the number of set bits among the M workers.
+ *
+ * Unless a function says otherwise:
+ *   - every pointer is a DEVICE pointer owned by the caller; the library does
+ *     not allocate, free or retain memory, and keeps no state between calls;
+ *   - float and word pointers must be 16-byte aligned; ld and ldw must be
+ *     multiples of 4 with ld >= d and ldw >= W (so every row is 16-byte
+ *     aligned); 1 <= M <= SSGD_MAX_WORKERS;
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream);
+ *     work is enqueued on it and the call returns without waiting;
+ *   - d == 0 is valid: nothing is launched, SSGD_OK is returned;
+ *   - buffers must not overlap except where "in place" is stated;
+ *   - arguments are checked on the host before anything is launched; a failed
+ *     check returns a status and touches no memory.  Nothing traps, aborts,
+ *     throws or prints.  Input values are not scanned (NaN/Inf follow the bit
+ *     rule above).
+ */
+#ifndef SIGNSGD_B200_H_
+#define SIGNSGD_B200_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define SSGD_MAX_WORKERS 1024
+
+typedef enum {
+  SSGD_OK = 0,
+  SSGD_ERR_NULL = 1,  /* a required pointer is NULL                            */
+  SSGD_ERR_ALIGN = 2, /* pointer not 16-byte aligned, or ld / ldw not 4-aligned */
+  SSGD_ERR_SIZE = 3,  /* M out of range, ld < d, ldw < W, or a size overflows   */
+  SSGD_ERR_ARG = 4,   /* beta outside [0,1) or NaN; delta not finite            */
+  SSGD_ERR_CUDA = 5   /* the CUDA runtime reported an error at launch / copy    */
+} ssgd_status;
+
+/* ceil(d / 32): words per packed sign vector (d bits per vector, Table 1). */
+size_t ssgd_words(size_t d);
+
+/* Static, NUL-terminated description of a status code. */
+const char* ssgd_status_str(ssgd_status s);
+
+/* Algorithm 1, second line, and Algorithm 3 "pull sign(g_m)": each worker's
+ * gradient becomes its 1-bit sign vector.
+ *   g    in   [M][ld] gradients
+ *   bits out  [M][ldw] packed signs, bit i of row w = !(g[w][i] < 0)          */
+ssgd_status ssgd_sign_pack(const float* g, size_t M, size_t d, size_t ld,
+                           uint32_t* bits, size_t ldw, void* stream);
+
+/* Algorithm 2, lines 2-3, per worker, fused with the sign packing: in place
+ *   m[w][i] <- fma(beta, m[w][i], fl((1 - beta) * g[w][i]))      (fp32, RN)
+ * and bit i of row w = !(m_new[w][i] < 0): the sign of the NEW momentum is
+ * what the worker sends.  beta in [0,1); beta == 0 gives m <- g and the bits
+ * of ssgd_sign_pack.
+ *   g    in      [M][ld]
+ *   m    in/out  [M][ld], updated in place (elements >= d untouched)
+ *   bits out     [M][ldw]                                                      */
+ssgd_status ssgd_signum_momentum_pack(const float* g, float* m, size_t M,
+                                      size_t d, size_t ld, float beta,
+                                      uint32_t* bits, size_t ldw, void* stream);
+
+/* Algorithm 3, server block: vote = sign[ sum_m sign(.) ] per parameter (the
+ * "(best)" update of Section 4), from the M packed rows.
+ *   bits in   [M][ldw]  (padding bits of each row must be 0, as written by the
+ *                        two calls above)
+ *   vote out  [W]       voted bit = [popcount over workers >= ceil(M/2)]       */
+ssgd_status ssgd_majority_vote(const uint32_t* bits, size_t M, size_t d,
+                               size_t ldw, uint32_t* vote, void* stream);
+
+/* Algorithm 3, worker block (and the last line of Algorithms 1 and 2):
+ *   x[i] <- x[i] - delta if voted bit i is 1, else x[i] + delta   (fp32, RN)
+ *   x    in/out [d], in place;  vote in [W];  delta finite.                    */
+ssgd_status ssgd_sign_apply(float* x, const uint32_t* vote, size_t d,
+                            float delta, void* stream);
+
+/* One whole step of Algorithm 3 with Signum workers: momentum + pack for all
+ * M workers, majority vote, apply; same results as the three calls above in
+ * sequence on `stream`.
+ *   x        in/out [d]
+ *   g        in     [M][ld]
+ *   m        in/out [M][ld]; may be NULL only when beta == 0, which selects
+ *                   Algorithm 3 as printed (workers send sign(g), no momentum)
+ *   bits_ws  out    [M][ldw] workspace: holds the workers' wire words on return
+ *   vote_ws  out    [W]      workspace: holds the server's wire words on return */
+ssgd_status ssgd_signsgd_step(float* x, const float* g, float* m, size_t M,
+                              size_t d, size_t ld, float beta, float delta,
+                              uint32_t* bits_ws, size_t ldw, uint32_t* vote_ws,
+                              void* stream);
+
+/* ssgd_signsgd_step for a caller whose gradients live in HOST memory
+ * (Algorithm 3's "independent gradient estimate" arriving from outside the
+ * device): copies g_host to the device staging buffer, runs the step, and
+ * copies the voted words back to the host, all enqueued on `stream`.
+ *   g_host    in   HOST  [M][ld]; page-locked memory makes the copy asynchronous
+ *   g_stage   out  DEVICE [M][ld] staging buffer for the gradients
+ *   vote_host out  HOST  [W] (may be NULL: no copy back); valid once `stream`
+ *                  has been synchronised
+ *   x, m, bits_ws, vote_ws: DEVICE, as in ssgd_signsgd_step.                   */
+ssgd_status ssgd_signsgd_step_host(float* x, const float* g_host, float* m,
+                                   size_t M, size_t d, size_t ld, float beta,
+                                   float delta, float* g_stage,
+                                   uint32_t* bits_ws, size_t ldw,
+                                   uint32_t* vote_ws, uint32_t* vote_host,
+                                   void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SIGNSGD_B200_H_ */

@@ -1,0 +1,168 @@
+"""Thin Python binding of the C ABI in ``include/signsgd.h``.
+
+Argument marshalling only: every function takes torch tensors (device memory
+and streams are torch's), checks dtype / device / contiguity, and passes raw
+pointers and sizes to the function of the same name in ``libsignsgd_b200.so``.
+All arithmetic of Algorithms 1-3 runs inside that library's CUDA kernels.
+There is no fallback: if the library is missing or a call fails, an exception
+is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libsignsgd_b200.so")
+MAX_WORKERS = 1024
+
+_lib = None
+
+
+class SignSGDError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__("%s failed: status %d (%s)" % (where, status, status_str(status)))
+
+
+def lib() -> ctypes.CDLL:
+    """Load the CUDA library (built by ``_build.build()``); raises if it is absent."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(
+            "%s not found: build it with `python -m paper_1802_04434_b200._build` "
+            "(needs nvcc); there is no CPU fallback" % LIB_PATH)
+    L = ctypes.CDLL(LIB_PATH)
+    sz, f32, vp, ci = ctypes.c_size_t, ctypes.c_float, ctypes.c_void_p, ctypes.c_int
+    L.ssgd_words.restype = sz
+    L.ssgd_words.argtypes = [sz]
+    L.ssgd_status_str.restype = ctypes.c_char_p
+    L.ssgd_status_str.argtypes = [ci]
+    sigs = {
+        "ssgd_sign_pack": [vp, sz, sz, sz, vp, sz, vp],
+        "ssgd_signum_momentum_pack": [vp, vp, sz, sz, sz, f32, vp, sz, vp],
+        "ssgd_majority_vote": [vp, sz, sz, sz, vp, vp],
+        "ssgd_sign_apply": [vp, vp, sz, f32, vp],
+        "ssgd_signsgd_step": [vp, vp, vp, sz, sz, sz, f32, f32, vp, sz, vp, vp],
+        "ssgd_signsgd_step_host": [vp, vp, vp, sz, sz, sz, f32, f32, vp, vp, sz, vp, vp, vp],
+    }
+    for name, args in sigs.items():
+        fn = getattr(L, name)
+        fn.restype = ci
+        fn.argtypes = args
+    _lib = L
+    return L
+
+
+def status_str(status: int) -> str:
+    return lib().ssgd_status_str(int(status)).decode()
+
+
+def words(d: int) -> int:
+    """ceil(d / 32)."""
+    return int(lib().ssgd_words(d))
+
+
+def _ptr(t: Optional[torch.Tensor], dtype, name: str, cuda: bool = True) -> Optional[int]:
+    if t is None:
+        return None
+    if not isinstance(t, torch.Tensor) or t.dtype != dtype:
+        raise TypeError("%s must be a torch tensor of dtype %s" % (name, dtype))
+    if t.is_cuda != cuda:
+        raise ValueError("%s must live in %s memory" % (name, "device" if cuda else "host"))
+    if not t.is_contiguous():
+        raise ValueError("%s must be contiguous" % name)
+    return t.data_ptr()
+
+
+def _need(t: torch.Tensor, n: int, name: str) -> None:
+    if t.numel() < n:
+        raise ValueError("%s holds %d elements, the call needs %d" % (name, t.numel(), n))
+
+
+def _stream(stream) -> int:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
+
+
+def _check(status: int, where: str) -> None:
+    if status != 0:
+        raise SignSGDError(status, where)
+
+
+# words are stored in int32 tensors on the torch side (torch has no full uint32 support);
+# the library sees the same 32 bits.
+WORD_DTYPE = torch.int32
+
+
+def sign_pack(g: torch.Tensor, M: int, d: int, ld: int, bits: torch.Tensor, ldw: int,
+              stream=None) -> None:
+    """Algorithm 1 / 3 worker side: bits[w] <- packed sign(g[w])."""
+    _need(g, M * ld, "g"); _need(bits, M * ldw, "bits")
+    _check(lib().ssgd_sign_pack(_ptr(g, torch.float32, "g"), M, d, ld,
+                                _ptr(bits, WORD_DTYPE, "bits"), ldw, _stream(stream)),
+           "ssgd_sign_pack")
+
+
+def signum_momentum_pack(g: torch.Tensor, m: torch.Tensor, M: int, d: int, ld: int, beta: float,
+                         bits: torch.Tensor, ldw: int, stream=None) -> None:
+    """Algorithm 2 per worker, fused with packing: m updated in place, bits <- sign(m_new)."""
+    _need(g, M * ld, "g"); _need(m, M * ld, "m"); _need(bits, M * ldw, "bits")
+    _check(lib().ssgd_signum_momentum_pack(
+        _ptr(g, torch.float32, "g"), _ptr(m, torch.float32, "m"), M, d, ld, beta,
+        _ptr(bits, WORD_DTYPE, "bits"), ldw, _stream(stream)), "ssgd_signum_momentum_pack")
+
+
+def majority_vote(bits: torch.Tensor, M: int, d: int, ldw: int, vote: torch.Tensor,
+                  stream=None) -> None:
+    """Algorithm 3 server side: vote <- packed sign of the sum of the workers' signs."""
+    _need(bits, M * ldw, "bits"); _need(vote, -(-d // 32), "vote")
+    _check(lib().ssgd_majority_vote(_ptr(bits, WORD_DTYPE, "bits"), M, d, ldw,
+                                    _ptr(vote, WORD_DTYPE, "vote"), _stream(stream)),
+           "ssgd_majority_vote")
+
+
+def sign_apply(x: torch.Tensor, vote: torch.Tensor, d: int, delta: float, stream=None) -> None:
+    """Algorithm 3 worker side: x <- x - delta * sign(vote), in place."""
+    _need(x, d, "x"); _need(vote, -(-d // 32), "vote")
+    _check(lib().ssgd_sign_apply(_ptr(x, torch.float32, "x"), _ptr(vote, WORD_DTYPE, "vote"), d,
+                                 delta, _stream(stream)), "ssgd_sign_apply")
+
+
+def signsgd_step(x: torch.Tensor, g: torch.Tensor, m: Optional[torch.Tensor], M: int, d: int,
+                 ld: int, beta: float, delta: float, bits_ws: torch.Tensor, ldw: int,
+                 vote_ws: torch.Tensor, stream=None) -> None:
+    """One step of Algorithm 3 with Signum workers (m=None with beta=0: plain signSGD)."""
+    _need(x, d, "x"); _need(g, M * ld, "g"); _need(bits_ws, M * ldw, "bits_ws")
+    _need(vote_ws, -(-d // 32), "vote_ws")
+    if m is not None:
+        _need(m, M * ld, "m")
+    _check(lib().ssgd_signsgd_step(
+        _ptr(x, torch.float32, "x"), _ptr(g, torch.float32, "g"), _ptr(m, torch.float32, "m"),
+        M, d, ld, beta, delta, _ptr(bits_ws, WORD_DTYPE, "bits_ws"), ldw,
+        _ptr(vote_ws, WORD_DTYPE, "vote_ws"), _stream(stream)), "ssgd_signsgd_step")
+
+
+def signsgd_step_host(x: torch.Tensor, g_host: torch.Tensor, m: Optional[torch.Tensor], M: int,
+                      d: int, ld: int, beta: float, delta: float, g_stage: torch.Tensor,
+                      bits_ws: torch.Tensor, ldw: int, vote_ws: torch.Tensor,
+                      vote_host: Optional[torch.Tensor], stream=None) -> None:
+    """The whole step with gradients in (pinned) host memory and the vote read back to the host."""
+    _need(x, d, "x"); _need(g_host, M * ld, "g_host"); _need(g_stage, M * ld, "g_stage")
+    _need(bits_ws, M * ldw, "bits_ws"); _need(vote_ws, -(-d // 32), "vote_ws")
+    if m is not None:
+        _need(m, M * ld, "m")
+    if vote_host is not None:
+        _need(vote_host, -(-d // 32), "vote_host")
+    _check(lib().ssgd_signsgd_step_host(
+        _ptr(x, torch.float32, "x"), _ptr(g_host, torch.float32, "g_host", cuda=False),
+        _ptr(m, torch.float32, "m"), M, d, ld, beta, delta,
+        _ptr(g_stage, torch.float32, "g_stage"), _ptr(bits_ws, WORD_DTYPE, "bits_ws"), ldw,
+        _ptr(vote_ws, WORD_DTYPE, "vote_ws"), _ptr(vote_host, WORD_DTYPE, "vote_host", cuda=False),
+        _stream(stream)), "ssgd_signsgd_step_host")

@@ -1,0 +1,566 @@
+// sm_100a kernels and C ABI for the signSGD / Signum / majority-vote step
+// (Algorithms 1-3 of Bernstein et al., "signSGD: Compressed Optimisation for
+// Non-Convex Problems").  See include/signsgd.h for the contract of each call.
+//
+// Every kernel here streams its operands once and is bound by HBM bandwidth:
+//   worker kernel   12.125 B per parameter per worker (g read, m read + write,
+//                   1/8 B of sign bits written); 4.125 B for the sign-only form
+//   vote kernel     (M + 1) / 8 B per parameter
+//   apply kernel    8.125 B per parameter
+// so the design rules are: 128-bit coalesced accesses, many independent loads
+// in flight per thread, streaming cache hints (nothing is re-read), grids sized
+// in whole waves of the SM count, and 64-bit indexing (M * d exceeds 2^32).
+
+#include <cuda_runtime.h>
+#include <math.h>
+#include <stdint.h>
+
+#include "signsgd.h"
+
+namespace {
+
+// ---------------------------------------------------------------------------
+// small device helpers
+
+// Streaming 128-bit accesses: the data is touched once, so it should neither
+// stay in L1 nor displace useful lines in L2.
+__device__ __forceinline__ float4 ld_stream(const float* p) {
+  return __ldcs(reinterpret_cast<const float4*>(p));
+}
+__device__ __forceinline__ void st_stream(float* p, float4 v) {
+  __stcs(reinterpret_cast<float4*>(p), v);
+}
+
+// sign(.) of Algorithms 1-3 in one bit: +0, -0 and NaN all count as +1.
+__device__ __forceinline__ unsigned sign_bit(float v) { return (v < 0.0f) ? 0u : 1u; }
+
+// Algorithm 2, second step, as two correctly rounded fp32 operations.  Written
+// with explicit intrinsics so that the compiler can neither contract nor split them.
+__device__ __forceinline__ float momentum_update(float beta, float omb, float m, float g) {
+  return __fmaf_rn(beta, m, __fmul_rn(omb, g));
+}
+
+// A warp holds 128 consecutive elements, lane l the four elements 4l..4l+3.
+// Lane l's four sign bits are bits 4(l%8)..4(l%8)+3 of word l/8, so an OR over
+// each group of eight lanes assembles the four canonical words; every lane of a
+// group receives its group's word.
+__device__ __forceinline__ unsigned assemble_word(unsigned nibble, unsigned lane) {
+  const unsigned group_mask = 0xFFu << (lane & 24u);
+  return __reduce_or_sync(group_mask, nibble << (4u * (lane & 7u)));
+}
+
+// ---------------------------------------------------------------------------
+// worker kernel: [momentum update +] sign + 1-bit pack, all M rows in one launch
+//
+// Work is cut into tiles of TILE = THREADS * 4 * UNROLL elements of one row.  A
+// warp owns 128 * UNROLL consecutive elements of the tile, so that the words it
+// produces are consecutive too.  Tiles are numbered row-major over (row, tile in
+// row) and dealt to CTAs round-robin.
+
+constexpr int kWorkerThreads = 256;
+
+template <bool MOMENTUM, int UNROLL>
+__global__ void __launch_bounds__(kWorkerThreads)
+worker_pack_kernel(const float* __restrict__ g, float* __restrict__ m,
+                   uint32_t* __restrict__ bits, unsigned long long d,
+                   unsigned long long ld, unsigned long long ldw,
+                   unsigned long long tiles_per_row, unsigned long long total_tiles,
+                   float beta, float omb) {
+  constexpr unsigned long long TILE = (unsigned long long)kWorkerThreads * 4 * UNROLL;
+  constexpr unsigned WARP_SPAN = 128 * UNROLL;
+  const unsigned lane = threadIdx.x & 31u;
+  const unsigned warp = threadIdx.x >> 5;
+
+  for (unsigned long long t = blockIdx.x; t < total_tiles; t += gridDim.x) {
+    const unsigned long long row = t / tiles_per_row;
+    const unsigned long long tile = t - row * tiles_per_row;
+    // first element of this warp's span, within the row
+    const unsigned long long e0 = tile * TILE + (unsigned long long)warp * WARP_SPAN;
+    if (e0 >= d) continue;
+    const float* gr = g + row * ld;
+    float* mr = MOMENTUM ? m + row * ld : nullptr;
+    uint32_t* br = bits + row * ldw + (e0 >> 5);
+
+    if (e0 + WARP_SPAN <= d) {
+      // interior: no bounds checks, all loads issued before any use
+      float4 gv[UNROLL], mv[UNROLL];
+#pragma unroll
+      for (int u = 0; u < UNROLL; ++u) gv[u] = ld_stream(gr + e0 + u * 128 + lane * 4);
+      if (MOMENTUM) {
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) mv[u] = ld_stream(mr + e0 + u * 128 + lane * 4);
+      }
+#pragma unroll
+      for (int u = 0; u < UNROLL; ++u) {
+        float4 v = gv[u];
+        if (MOMENTUM) {
+          v.x = momentum_update(beta, omb, mv[u].x, v.x);
+          v.y = momentum_update(beta, omb, mv[u].y, v.y);
+          v.z = momentum_update(beta, omb, mv[u].z, v.z);
+          v.w = momentum_update(beta, omb, mv[u].w, v.w);
+          st_stream(mr + e0 + u * 128 + lane * 4, v);
+        }
+        const unsigned nib = sign_bit(v.x) | (sign_bit(v.y) << 1) | (sign_bit(v.z) << 2) |
+                             (sign_bit(v.w) << 3);
+        const unsigned word = assemble_word(nib, lane);
+        if ((lane & 7u) == 0) br[u * 4 + (lane >> 3)] = word;
+      }
+    } else {
+      // ragged end of the row: element-wise guards, padding bits stay 0, and
+      // nothing at or beyond d is written
+#pragma unroll 1
+      for (int u = 0; u < UNROLL; ++u) {
+        const unsigned long long e = e0 + u * 128 + lane * 4;
+        unsigned nib = 0;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          if (e + k < d) {
+            float v = gr[e + k];
+            if (MOMENTUM) {
+              v = momentum_update(beta, omb, mr[e + k], v);
+              mr[e + k] = v;
+            }
+            nib |= sign_bit(v) << k;
+          }
+        }
+        const unsigned word = assemble_word(nib, lane);
+        const unsigned long long first = e0 + u * 128 + (lane >> 3) * 32;  // first element of the word
+        if ((lane & 7u) == 0 && first < d) br[u * 4 + (lane >> 3)] = word;
+      }
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------
+// majority vote: bit-sliced vertical counter
+//
+// One thread owns four consecutive words (128 parameters) and walks down the M
+// rows.  The count of set bits per parameter is kept as NP bit-planes (plane p
+// holds bit p of all 128 counters), and rows are folded in with carry-save
+// adders (3 words in, sum + carry out: one XOR3 and one MAJ3 per word), eight
+// rows per block, so the cost is about two logic operations per input word.
+//
+// The comparison with the threshold T = ceil(M/2) is folded into the counter's
+// start value: with L = NP - 1 chosen so that floor(M/2) < 2^L, the counter
+// starts at 2^L - T and can reach at most 2^L - T + M < 2^(L+1); its top plane
+// is then exactly [P >= T], the voted bit (ties, 2P = M, included).
+
+struct W4 {
+  unsigned x, y, z, w;
+};
+__device__ __forceinline__ W4 ld_words(const uint32_t* p) {
+  const uint4 v = __ldcs(reinterpret_cast<const uint4*>(p));
+  return W4{v.x, v.y, v.z, v.w};
+}
+__device__ __forceinline__ unsigned xor3(unsigned a, unsigned b, unsigned c) { return a ^ b ^ c; }
+__device__ __forceinline__ unsigned maj3(unsigned a, unsigned b, unsigned c) {
+  return (a & b) | (c & (a | b));
+}
+// carry-save adder on 4 words: lo <- a ^ b ^ lo, returns the carries
+__device__ __forceinline__ W4 csa(W4& lo, const W4& a, const W4& b) {
+  W4 hi{maj3(lo.x, a.x, b.x), maj3(lo.y, a.y, b.y), maj3(lo.z, a.z, b.z), maj3(lo.w, a.w, b.w)};
+  lo = W4{xor3(lo.x, a.x, b.x), xor3(lo.y, a.y, b.y), xor3(lo.z, a.z, b.z), xor3(lo.w, a.w, b.w)};
+  return hi;
+}
+
+template <int NP>
+struct Counter {
+  W4 c[NP];
+  // add a word of weight 2^K: ripple from plane K upwards
+  template <int K>
+  __device__ __forceinline__ void add(W4 v) {
+#pragma unroll
+    for (int p = K; p < NP; ++p) {
+      const W4 carry{c[p].x & v.x, c[p].y & v.y, c[p].z & v.z, c[p].w & v.w};
+      c[p] = W4{c[p].x ^ v.x, c[p].y ^ v.y, c[p].z ^ v.z, c[p].w ^ v.w};
+      v = carry;
+    }
+  }
+  __device__ __forceinline__ void add2(const W4& a, const W4& b) {
+    if (NP >= 2) {
+      const W4 h = csa(c[0], a, b);
+      add<1>(h);
+    }
+  }
+  __device__ __forceinline__ void add4(const W4* a) {
+    if (NP >= 3) {
+      const W4 hA = csa(c[0], a[0], a[1]);
+      const W4 hB = csa(c[0], a[2], a[3]);
+      const W4 q = csa(c[1], hA, hB);
+      add<2>(q);
+    }
+  }
+  __device__ __forceinline__ void add8(const W4* a) {
+    if (NP >= 4) {
+      const W4 hA = csa(c[0], a[0], a[1]);
+      const W4 hB = csa(c[0], a[2], a[3]);
+      const W4 qA = csa(c[1], hA, hB);
+      const W4 hC = csa(c[0], a[4], a[5]);
+      const W4 hD = csa(c[0], a[6], a[7]);
+      const W4 qB = csa(c[1], hC, hD);
+      const W4 e = csa(c[2], qA, qB);
+      add<3>(e);
+    }
+  }
+};
+
+constexpr int kVoteThreads = 256;
+
+template <int NP>
+__global__ void __launch_bounds__(kVoteThreads)
+vote_kernel(const uint32_t* __restrict__ bits, unsigned M, unsigned long long d,
+            unsigned long long W, unsigned long long ldw, uint32_t* __restrict__ vote,
+            unsigned start_value) {
+  const unsigned long long chunks = (W + 3) / 4;
+  const unsigned long long stride = (unsigned long long)gridDim.x * kVoteThreads;
+  for (unsigned long long q = (unsigned long long)blockIdx.x * kVoteThreads + threadIdx.x;
+       q < chunks; q += stride) {
+    const uint32_t* col = bits + 4 * q;
+    Counter<NP> cnt;
+#pragma unroll
+    for (int p = 0; p < NP; ++p) {
+      const unsigned f = ((start_value >> p) & 1u) ? 0xFFFFFFFFu : 0u;
+      cnt.c[p] = W4{f, f, f, f};
+    }
+    unsigned w = 0;
+    if (NP >= 4) {
+      for (; w + 8 <= M; w += 8) {
+        W4 a[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) a[k] = ld_words(col + (unsigned long long)(w + k) * ldw);
+        cnt.add8(a);
+      }
+    }
+    if (NP >= 3 && w + 4 <= M) {
+      W4 a[4];
+#pragma unroll
+      for (int k = 0; k < 4; ++k) a[k] = ld_words(col + (unsigned long long)(w + k) * ldw);
+      cnt.add4(a);
+      w += 4;
+    }
+    if (NP >= 2 && w + 2 <= M) {
+      const W4 a = ld_words(col + (unsigned long long)w * ldw);
+      const W4 b = ld_words(col + (unsigned long long)(w + 1) * ldw);
+      cnt.add2(a, b);
+      w += 2;
+    }
+    if (w < M) {
+      cnt.template add<0>(ld_words(col + (unsigned long long)w * ldw));
+      w += 1;
+    }
+    W4 v = cnt.c[NP - 1];
+    // bits at positions >= d are written as 0, whatever the rows held there
+    const unsigned long long first = q * 128;  // first parameter of this chunk
+    unsigned out[4] = {v.x, v.y, v.z, v.w};
+    if (first + 128 <= d) {
+      *reinterpret_cast<uint4*>(vote + 4 * q) = make_uint4(out[0], out[1], out[2], out[3]);
+    } else {
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const unsigned long long lo = first + 32ull * k;
+        if (lo < d) {
+          const unsigned long long left = d - lo;
+          const unsigned mask = left >= 32 ? 0xFFFFFFFFu : ((1u << left) - 1u);
+          vote[4 * q + k] = out[k] & mask;
+        }
+      }
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------
+// apply: x <- x -/+ delta by the voted bit.  Thread layout as in the worker
+// kernel: lane l of a warp holds elements 4l..4l+3 of a 128-element span, whose
+// four bits sit at position 4(l%8) of word l/8 of the span.
+
+constexpr int kApplyThreads = 256;
+
+template <int UNROLL>
+__global__ void __launch_bounds__(kApplyThreads)
+apply_kernel(float* __restrict__ x, const uint32_t* __restrict__ vote, unsigned long long d,
+             unsigned long long total_tiles, float delta) {
+  constexpr unsigned long long TILE = (unsigned long long)kApplyThreads * 4 * UNROLL;
+  constexpr unsigned WARP_SPAN = 128 * UNROLL;
+  const unsigned lane = threadIdx.x & 31u;
+  const unsigned warp = threadIdx.x >> 5;
+  const float minus = -delta;
+  for (unsigned long long t = blockIdx.x; t < total_tiles; t += gridDim.x) {
+    const unsigned long long e0 = t * TILE + (unsigned long long)warp * WARP_SPAN;
+    if (e0 >= d) continue;
+    const uint32_t* vw = vote + (e0 >> 5);
+    if (e0 + WARP_SPAN <= d) {
+      float4 xv[UNROLL];
+      unsigned wv[UNROLL];
+#pragma unroll
+      for (int u = 0; u < UNROLL; ++u) {
+        xv[u] = ld_stream(x + e0 + u * 128 + lane * 4);
+        wv[u] = __ldg(vw + u * 4 + (lane >> 3));
+      }
+#pragma unroll
+      for (int u = 0; u < UNROLL; ++u) {
+        const unsigned nib = wv[u] >> (4u * (lane & 7u));
+        float4 v = xv[u];
+        v.x = __fadd_rn(v.x, (nib & 1u) ? minus : delta);
+        v.y = __fadd_rn(v.y, (nib & 2u) ? minus : delta);
+        v.z = __fadd_rn(v.z, (nib & 4u) ? minus : delta);
+        v.w = __fadd_rn(v.w, (nib & 8u) ? minus : delta);
+        st_stream(x + e0 + u * 128 + lane * 4, v);
+      }
+    } else {
+#pragma unroll 1
+      for (int u = 0; u < UNROLL; ++u) {
+        const unsigned long long e = e0 + u * 128 + lane * 4;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          if (e + k < d) {
+            const unsigned bit = (vote[(e + k) >> 5] >> ((e + k) & 31u)) & 1u;
+            x[e + k] = __fadd_rn(x[e + k], bit ? minus : delta);
+          }
+        }
+      }
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------
+// host side
+
+struct DeviceInfo {
+  int sms;
+};
+
+bool device_info(DeviceInfo* out) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return false;
+  static int cached_sms[64] = {0};
+  if (dev < 0 || dev >= 64) return false;
+  if (cached_sms[dev] == 0) {
+    int sms = 0;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
+      return false;
+    cached_sms[dev] = sms;
+  }
+  out->sms = cached_sms[dev];
+  return true;
+}
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+inline bool mul_overflows(size_t a, size_t b) { return b != 0 && a > SIZE_MAX / b; }
+
+ssgd_status check_rows(size_t M, size_t d, size_t ld, size_t ldw, bool need_ld) {
+  if (M < 1 || M > SSGD_MAX_WORKERS) return SSGD_ERR_SIZE;
+  if (d > SIZE_MAX - 31) return SSGD_ERR_SIZE;
+  const size_t W = ssgd_words(d);
+  if (need_ld) {
+    if (ld % 4 != 0) return SSGD_ERR_ALIGN;
+    if (ld < d || mul_overflows(M, ld) || mul_overflows(M * ld, sizeof(float))) return SSGD_ERR_SIZE;
+  }
+  if (ldw % 4 != 0) return SSGD_ERR_ALIGN;
+  if (ldw < W || mul_overflows(M, ldw) || mul_overflows(M * ldw, sizeof(uint32_t))) return SSGD_ERR_SIZE;
+  return SSGD_OK;
+}
+
+inline bool beta_ok(float beta) { return beta >= 0.0f && beta < 1.0f; }  // false for NaN
+
+ssgd_status launch_status() { return cudaGetLastError() == cudaSuccess ? SSGD_OK : SSGD_ERR_CUDA; }
+
+constexpr int kWorkerUnroll = 4;
+constexpr int kApplyUnroll = 4;
+
+unsigned grid_for(unsigned long long work_items, int sms, int ctas_per_sm) {
+  const unsigned long long full = (unsigned long long)sms * ctas_per_sm;
+  return (unsigned)(work_items < full ? work_items : full);
+}
+
+template <bool MOMENTUM>
+ssgd_status launch_worker(const float* g, float* m, size_t M, size_t d, size_t ld, float beta,
+                          uint32_t* bits, size_t ldw, cudaStream_t s) {
+  DeviceInfo di;
+  if (!device_info(&di)) return SSGD_ERR_CUDA;
+  constexpr unsigned long long TILE = (unsigned long long)kWorkerThreads * 4 * kWorkerUnroll;
+  const unsigned long long tiles_per_row = (d + TILE - 1) / TILE;
+  const unsigned long long total = tiles_per_row * M;
+  const unsigned grid = grid_for(total, di.sms, 8);
+  const float omb = 1.0f - beta;
+  worker_pack_kernel<MOMENTUM, kWorkerUnroll><<<grid, kWorkerThreads, 0, s>>>(
+      g, m, bits, d, ld, ldw, tiles_per_row, total, beta, omb);
+  return launch_status();
+}
+
+unsigned vote_planes(size_t M) {
+  unsigned L = 0;
+  while ((M / 2) >= (size_t(1) << L)) ++L;  // smallest L with floor(M/2) < 2^L
+  return L + 1;
+}
+
+template <int NP>
+void launch_vote_np(const uint32_t* bits, size_t M, size_t d, size_t W, size_t ldw, uint32_t* vote,
+                    unsigned grid, cudaStream_t s) {
+  const unsigned T = (unsigned)((M + 1) / 2);
+  const unsigned start = (1u << (NP - 1)) - T;
+  vote_kernel<NP><<<grid, kVoteThreads, 0, s>>>(bits, (unsigned)M, d, W, ldw, vote, start);
+}
+
+ssgd_status launch_vote(const uint32_t* bits, size_t M, size_t d, size_t ldw, uint32_t* vote,
+                        cudaStream_t s) {
+  DeviceInfo di;
+  if (!device_info(&di)) return SSGD_ERR_CUDA;
+  const size_t W = ssgd_words(d);
+  const unsigned long long chunks = (W + 3) / 4;
+  const unsigned long long ctas = (chunks + kVoteThreads - 1) / kVoteThreads;
+  const unsigned grid = grid_for(ctas, di.sms, 8);
+  switch (vote_planes(M)) {
+    case 1: launch_vote_np<1>(bits, M, d, W, ldw, vote, grid, s); break;
+    case 2: launch_vote_np<2>(bits, M, d, W, ldw, vote, grid, s); break;
+    case 3: launch_vote_np<3>(bits, M, d, W, ldw, vote, grid, s); break;
+    case 4: launch_vote_np<4>(bits, M, d, W, ldw, vote, grid, s); break;
+    case 5: launch_vote_np<5>(bits, M, d, W, ldw, vote, grid, s); break;
+    case 6: launch_vote_np<6>(bits, M, d, W, ldw, vote, grid, s); break;
+    case 7: launch_vote_np<7>(bits, M, d, W, ldw, vote, grid, s); break;
+    case 8: launch_vote_np<8>(bits, M, d, W, ldw, vote, grid, s); break;
+    case 9: launch_vote_np<9>(bits, M, d, W, ldw, vote, grid, s); break;
+    case 10: launch_vote_np<10>(bits, M, d, W, ldw, vote, grid, s); break;
+    case 11: launch_vote_np<11>(bits, M, d, W, ldw, vote, grid, s); break;
+    default: return SSGD_ERR_SIZE;
+  }
+  return launch_status();
+}
+
+ssgd_status launch_apply(float* x, const uint32_t* vote, size_t d, float delta, cudaStream_t s) {
+  DeviceInfo di;
+  if (!device_info(&di)) return SSGD_ERR_CUDA;
+  constexpr unsigned long long TILE = (unsigned long long)kApplyThreads * 4 * kApplyUnroll;
+  const unsigned long long total = (d + TILE - 1) / TILE;
+  const unsigned grid = grid_for(total, di.sms, 8);
+  apply_kernel<kApplyUnroll><<<grid, kApplyThreads, 0, s>>>(x, vote, d, total, delta);
+  return launch_status();
+}
+
+// argument checks shared by the entry points -------------------------------
+
+ssgd_status check_sign_pack(const float* g, size_t M, size_t d, size_t ld, const uint32_t* bits,
+                            size_t ldw) {
+  if (!g || !bits) return SSGD_ERR_NULL;
+  if (!aligned16(g) || !aligned16(bits)) return SSGD_ERR_ALIGN;
+  return check_rows(M, d, ld, ldw, true);
+}
+
+ssgd_status check_momentum_pack(const float* g, const float* m, size_t M, size_t d, size_t ld,
+                                float beta, const uint32_t* bits, size_t ldw) {
+  if (!g || !m || !bits) return SSGD_ERR_NULL;
+  if (!aligned16(g) || !aligned16(m) || !aligned16(bits)) return SSGD_ERR_ALIGN;
+  const ssgd_status st = check_rows(M, d, ld, ldw, true);
+  if (st != SSGD_OK) return st;
+  return beta_ok(beta) ? SSGD_OK : SSGD_ERR_ARG;
+}
+
+ssgd_status check_vote(const uint32_t* bits, size_t M, size_t d, size_t ldw, const uint32_t* vote) {
+  if (!bits || !vote) return SSGD_ERR_NULL;
+  if (!aligned16(bits) || !aligned16(vote)) return SSGD_ERR_ALIGN;
+  return check_rows(M, d, 0, ldw, false);
+}
+
+ssgd_status check_apply(const float* x, const uint32_t* vote, size_t d, float delta) {
+  if (!x || !vote) return SSGD_ERR_NULL;
+  if (!aligned16(x) || !aligned16(vote)) return SSGD_ERR_ALIGN;
+  if (d > SIZE_MAX - 31) return SSGD_ERR_SIZE;
+  return isfinite(delta) ? SSGD_OK : SSGD_ERR_ARG;
+}
+
+ssgd_status check_step(const float* x, const float* g, const float* m, size_t M, size_t d, size_t ld,
+                       float beta, float delta, const uint32_t* bits_ws, size_t ldw,
+                       const uint32_t* vote_ws) {
+  if (!x || !g || !bits_ws || !vote_ws) return SSGD_ERR_NULL;
+  if (!beta_ok(beta)) return SSGD_ERR_ARG;
+  if (!m && beta != 0.0f) return SSGD_ERR_NULL;
+  ssgd_status st = m ? check_momentum_pack(g, m, M, d, ld, beta, bits_ws, ldw)
+                     : check_sign_pack(g, M, d, ld, bits_ws, ldw);
+  if (st != SSGD_OK) return st;
+  st = check_vote(bits_ws, M, d, ldw, vote_ws);
+  if (st != SSGD_OK) return st;
+  return check_apply(x, vote_ws, d, delta);
+}
+
+}  // namespace
+
+// ---------------------------------------------------------------------------
+// C ABI
+
+extern "C" {
+
+size_t ssgd_words(size_t d) { return d / 32 + (d % 32 != 0 ? 1 : 0); }
+
+const char* ssgd_status_str(ssgd_status s) {
+  switch (s) {
+    case SSGD_OK: return "ok";
+    case SSGD_ERR_NULL: return "a required pointer is NULL";
+    case SSGD_ERR_ALIGN: return "pointer not 16-byte aligned or row stride not a multiple of 4";
+    case SSGD_ERR_SIZE: return "worker count out of range, row stride too short, or size overflow";
+    case SSGD_ERR_ARG: return "beta outside [0,1) or delta not finite";
+    case SSGD_ERR_CUDA: return "CUDA runtime error";
+  }
+  return "unknown status";
+}
+
+ssgd_status ssgd_sign_pack(const float* g, size_t M, size_t d, size_t ld, uint32_t* bits,
+                           size_t ldw, void* stream) {
+  const ssgd_status st = check_sign_pack(g, M, d, ld, bits, ldw);
+  if (st != SSGD_OK || d == 0) return st;
+  return launch_worker<false>(g, nullptr, M, d, ld, 0.0f, bits, ldw, static_cast<cudaStream_t>(stream));
+}
+
+ssgd_status ssgd_signum_momentum_pack(const float* g, float* m, size_t M, size_t d, size_t ld,
+                                      float beta, uint32_t* bits, size_t ldw, void* stream) {
+  const ssgd_status st = check_momentum_pack(g, m, M, d, ld, beta, bits, ldw);
+  if (st != SSGD_OK || d == 0) return st;
+  return launch_worker<true>(g, m, M, d, ld, beta, bits, ldw, static_cast<cudaStream_t>(stream));
+}
+
+ssgd_status ssgd_majority_vote(const uint32_t* bits, size_t M, size_t d, size_t ldw,
+                               uint32_t* vote, void* stream) {
+  const ssgd_status st = check_vote(bits, M, d, ldw, vote);
+  if (st != SSGD_OK || d == 0) return st;
+  return launch_vote(bits, M, d, ldw, vote, static_cast<cudaStream_t>(stream));
+}
+
+ssgd_status ssgd_sign_apply(float* x, const uint32_t* vote, size_t d, float delta, void* stream) {
+  const ssgd_status st = check_apply(x, vote, d, delta);
+  if (st != SSGD_OK || d == 0) return st;
+  return launch_apply(x, vote, d, delta, static_cast<cudaStream_t>(stream));
+}
+
+ssgd_status ssgd_signsgd_step(float* x, const float* g, float* m, size_t M, size_t d, size_t ld,
+                              float beta, float delta, uint32_t* bits_ws, size_t ldw,
+                              uint32_t* vote_ws, void* stream) {
+  ssgd_status st = check_step(x, g, m, M, d, ld, beta, delta, bits_ws, ldw, vote_ws);
+  if (st != SSGD_OK || d == 0) return st;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  st = m ? launch_worker<true>(g, m, M, d, ld, beta, bits_ws, ldw, s)
+         : launch_worker<false>(g, nullptr, M, d, ld, 0.0f, bits_ws, ldw, s);
+  if (st != SSGD_OK) return st;
+  st = launch_vote(bits_ws, M, d, ldw, vote_ws, s);
+  if (st != SSGD_OK) return st;
+  return launch_apply(x, vote_ws, d, delta, s);
+}
+
+ssgd_status ssgd_signsgd_step_host(float* x, const float* g_host, float* m, size_t M, size_t d,
+                                   size_t ld, float beta, float delta, float* g_stage,
+                                   uint32_t* bits_ws, size_t ldw, uint32_t* vote_ws,
+                                   uint32_t* vote_host, void* stream) {
+  if (!g_host) return SSGD_ERR_NULL;
+  ssgd_status st = check_step(x, g_stage, m, M, d, ld, beta, delta, bits_ws, ldw, vote_ws);
+  if (st != SSGD_OK || d == 0) return st;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (cudaMemcpyAsync(g_stage, g_host, M * ld * sizeof(float), cudaMemcpyHostToDevice, s) != cudaSuccess)
+    return SSGD_ERR_CUDA;
+  st = ssgd_signsgd_step(x, g_stage, m, M, d, ld, beta, delta, bits_ws, ldw, vote_ws, stream);
+  if (st != SSGD_OK) return st;
+  if (vote_host &&
+      cudaMemcpyAsync(vote_host, vote_ws, ssgd_words(d) * sizeof(uint32_t), cudaMemcpyDeviceToHost, s) !=
+          cudaSuccess)
+    return SSGD_ERR_CUDA;
+  return SSGD_OK;
+}
+
+}  // extern "C"

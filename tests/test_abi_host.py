@@ -1,0 +1,116 @@
+"""Host-side checks of the C ABI that need no GPU: the library loads, exports every
+symbol the header declares, and rejects bad arguments before launching anything."""
+import ctypes
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+HEADER = os.path.join(ROOT, "include", "signsgd.h")
+
+
+@pytest.fixture(scope="module")
+def L():
+    from paper_1802_04434_b200 import _build, binding
+    _build.build()
+    return binding.lib()
+
+
+def declared_symbols():
+    text = open(HEADER).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(ssgd_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_header_declares_the_expected_calls():
+    names = declared_symbols()
+    for n in ("ssgd_sign_pack", "ssgd_signum_momentum_pack", "ssgd_majority_vote", "ssgd_sign_apply",
+              "ssgd_signsgd_step", "ssgd_words", "ssgd_status_str"):
+        assert n in names
+
+
+def test_library_exports_every_declared_symbol(L):
+    for n in declared_symbols():
+        assert hasattr(L, n), n
+
+
+def test_words(L):
+    for d in (0, 1, 31, 32, 33, 25_557_056, 335_141_888, 2**40 + 1):
+        assert L.ssgd_words(d) == -(-d // 32)
+
+
+def test_status_strings(L):
+    seen = {L.ssgd_status_str(i) for i in range(6)}
+    assert len(seen) == 6 and all(s for s in seen)
+
+
+A = 0x10000          # a fake, 16-byte aligned address: these calls must fail before touching it
+OK, NULL, ALIGN, SIZE, ARG = 0, 1, 2, 3, 4
+
+
+def test_sign_pack_argument_checks(L):
+    f = L.ssgd_sign_pack
+    assert f(None, 1, 64, 64, A, 4, None) == NULL
+    assert f(A, 1, 64, 64, None, 4, None) == NULL
+    assert f(A + 4, 1, 64, 64, A, 4, None) == ALIGN
+    assert f(A, 1, 64, 64, A + 8, 4, None) == ALIGN
+    assert f(A, 1, 64, 66, A, 4, None) == ALIGN            # ld not a multiple of 4
+    assert f(A, 1, 64, 64, A, 2, None) == ALIGN            # ldw not a multiple of 4
+    assert f(A, 0, 64, 64, A, 4, None) == SIZE             # M = 0
+    assert f(A, 1025, 64, 64, A, 4, None) == SIZE          # M above the maximum
+    assert f(A, 1, 64, 60, A, 4, None) == SIZE             # ld < d
+    assert f(A, 1, 160, 160, A, 4, None) == SIZE           # ldw < W = 5
+    assert f(A, 4, 2**62, 2**62, A, 2**57, None) == SIZE   # M * ld overflows
+    assert f(A, 1, 0, 0, A, 0, None) == OK                 # d = 0: nothing to do
+
+
+def test_momentum_pack_argument_checks(L):
+    f = L.ssgd_signum_momentum_pack
+    assert f(A, None, 1, 64, 64, 0.9, A, 4, None) == NULL
+    assert f(A, A + 4, 1, 64, 64, 0.9, A, 4, None) == ALIGN
+    for beta in (1.0, 1.5, -0.1, float("nan"), float("inf")):
+        assert f(A, A, 1, 64, 64, beta, A, 4, None) == ARG
+    assert f(A, A, 1, 0, 0, 0.0, A, 0, None) == OK
+
+
+def test_vote_argument_checks(L):
+    f = L.ssgd_majority_vote
+    assert f(None, 3, 64, 4, A, None) == NULL
+    assert f(A, 3, 64, 4, None, None) == NULL
+    assert f(A, 3, 64, 4, A + 4, None) == ALIGN
+    assert f(A, 3, 64, 6, A, None) == ALIGN
+    assert f(A, 0, 64, 4, A, None) == SIZE
+    assert f(A, 3, 640, 16, A, None) == SIZE               # W = 20 > ldw
+    assert f(A, 3, 0, 0, A, None) == OK
+
+
+def test_apply_argument_checks(L):
+    f = L.ssgd_sign_apply
+    assert f(None, A, 64, 0.1, None) == NULL
+    assert f(A, None, 64, 0.1, None) == NULL
+    assert f(A + 4, A, 64, 0.1, None) == ALIGN
+    for delta in (float("nan"), float("inf"), float("-inf")):
+        assert f(A, A, 64, delta, None) == ARG
+    assert f(A, A, 0, 0.1, None) == OK
+
+
+def test_step_argument_checks(L):
+    f = L.ssgd_signsgd_step
+    assert f(None, A, A, 1, 64, 64, 0.9, 0.1, A, 4, A, None) == NULL
+    assert f(A, A, None, 1, 64, 64, 0.9, 0.1, A, 4, A, None) == NULL     # m required when beta > 0
+    assert f(A, A, None, 1, 0, 0, 0.0, 0.1, A, 0, A, None) == OK         # m optional when beta = 0
+    assert f(A, A, A, 1, 64, 64, 1.0, 0.1, A, 4, A, None) == ARG
+    assert f(A, A, A, 1, 64, 64, 0.9, float("nan"), A, 4, A, None) == ARG
+    assert f(A, A, A, 2000, 64, 64, 0.9, 0.1, A, 4, A, None) == SIZE
+    h = L.ssgd_signsgd_step_host
+    assert h(A, None, A, 1, 64, 64, 0.9, 0.1, A, A, 4, A, None, None) == NULL
+    assert h(A, A, A, 1, 64, 64, 0.9, 0.1, A + 4, A, 4, A, None, None) == ALIGN
+
+
+def test_binding_refuses_to_run_without_the_library(monkeypatch, tmp_path):
+    from paper_1802_04434_b200 import binding
+    monkeypatch.setattr(binding, "_lib", None)
+    monkeypatch.setattr(binding, "LIB_PATH", str(tmp_path / "missing.so"))
+    with pytest.raises(ImportError):
+        binding.words(64)

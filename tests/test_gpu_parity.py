@@ -1,0 +1,342 @@
+"""GPU parity: every entry point of the C ABI against the CPU oracle, element by
+element on the same seeded inputs.
+
+Acceptance (stated by the task's target and derived from the arithmetic): packed
+sign words and vote words bit-exact; m and x within 1 ulp of fp32
+(|diff| <= 1.2e-7 * |value|).  Both sides evaluate the momentum as the same two
+correctly rounded fp32 operations and the apply step as one correctly rounded
+add, so the tests below demand equality of the fp32 bit patterns, which is
+stricter; a sign bit may therefore never differ either.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_1802_04434_b200 import binding as B
+from paper_1802_04434_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+DEV = "cuda:0"
+CANARY_WORD = -559038737  # 0xDEADBEEF as int32
+CANARY_F = 12345.678
+
+
+def u32(t: torch.Tensor) -> np.ndarray:
+    return t.detach().cpu().numpy().view(np.uint32)
+
+
+def f32(t: torch.Tensor) -> np.ndarray:
+    return t.detach().cpu().numpy()
+
+
+def assert_same_f32(a: np.ndarray, b: np.ndarray, what: str):
+    """Bit-identical fp32 (NaN payloads aside); reports the 1-ulp acceptance bound on failure."""
+    ai, bi = a.view(np.uint32), b.view(np.uint32)
+    same = (ai == bi) | (np.isnan(a) & np.isnan(b))
+    if not same.all():
+        bad = np.flatnonzero(~same)
+        i = bad[0]
+        rel = abs(float(a[i]) - float(b[i])) / max(abs(float(b[i])), 1e-45)
+        raise AssertionError("%s: %d of %d elements differ, first at %d: gpu %r oracle %r (rel %.3g; "
+                             "acceptance bound 1.2e-7)" % (what, bad.size, a.size, i, a[i], b[i], rel))
+
+
+def rand_inputs(M, d, ld, seed, special=False):
+    r = np.random.default_rng(seed)
+    g = (r.standard_normal((M, ld)) * 10.0 ** r.integers(-3, 2, (M, ld))).astype(np.float32)
+    m = (r.standard_normal((M, ld)) * 10.0 ** r.integers(-3, 2, (M, ld))).astype(np.float32)
+    x = r.standard_normal(max(d, 1)).astype(np.float32)
+    g[r.random((M, ld)) < 0.03] = 0.0
+    if special and d >= 16:
+        vals = np.array([0.0, -0.0, np.nan, np.inf, -np.inf, 1e-45, -1e-45, 1e-39, -1e-39,
+                         3.4e38, -3.4e38, 1.17549435e-38], dtype=np.float32)
+        for w in range(M):
+            idx = r.choice(d, size=min(d, 24), replace=False)
+            g[w, idx] = r.choice(vals, size=idx.size)
+            idx = r.choice(d, size=min(d, 24), replace=False)
+            m[w, idx] = r.choice(vals, size=idx.size)
+    return g, m, x
+
+
+SMALL_D = [1, 2, 31, 32, 33, 127, 128, 129, 511, 512, 513, 4095, 4096, 4097, 5000, 16389, 100003]
+SMALL_M = [1, 2, 3, 4, 7, 8, 15, 16, 31, 32, 33]
+
+
+@pytest.mark.parametrize("d", SMALL_D)
+def test_sign_pack_and_momentum_pack_small(d):
+    for M in (1, 3, 8):
+        ld = wl.round_up(d, 4) + 4
+        W = oracle.words(d)
+        ldw = wl.round_up(W, 4) + 4
+        g, m, _ = rand_inputs(M, d, ld, seed=d * 31 + M, special=True)
+        gd = torch.from_numpy(g).to(DEV)
+        # sign_pack
+        bits = torch.full((M, ldw), CANARY_WORD, dtype=torch.int32, device=DEV)
+        B.sign_pack(gd, M, d, ld, bits, ldw)
+        ref = oracle.sign_pack(g.reshape(-1), M, d, ld=ld, ldw=ldw).reshape(M, ldw)
+        got = u32(bits)
+        assert np.array_equal(got[:, :W], ref[:, :W])
+        assert np.all(got[:, W:] == np.uint32(0xDEADBEEF))      # row padding never written
+        # signum_momentum_pack
+        for beta in (0.9, 0.0):
+            md = torch.from_numpy(m).to(DEV)
+            bits.fill_(CANARY_WORD)
+            B.signum_momentum_pack(gd, md, M, d, ld, beta, bits, ldw)
+            m_ref = m.copy().reshape(-1)
+            ref = oracle.signum_momentum_pack(g.reshape(-1), m_ref, M, d, beta, ld=ld, ldw=ldw).reshape(M, ldw)
+            got_m = f32(md)
+            assert_same_f32(got_m.reshape(-1), m_ref, "m (d=%d M=%d beta=%g)" % (d, M, beta))
+            assert np.array_equal(got_m[:, d:].view(np.uint32), m[:, d:].view(np.uint32))
+            got = u32(bits)
+            assert np.array_equal(got[:, :W], ref[:, :W])
+            assert np.all(got[:, W:] == np.uint32(0xDEADBEEF))
+
+
+@pytest.mark.parametrize("M", SMALL_M + [64, 100, 255, 256, 1000, 1024])
+def test_majority_vote_small(M):
+    for d in (1, 33, 128, 1000, 4097, 40000 if M <= 64 else 3000):
+        r = np.random.default_rng(M * 1000 + d)
+        W = oracle.words(d)
+        ldw = wl.round_up(W, 4) + (4 if M % 2 else 0)
+        p = r.random(d) if M > 2 else np.full(d, 0.5)           # per-element bias: spans all counts
+        s = (r.random((M, d)) < p).astype(np.uint8)
+        rows = np.zeros((M, ldw), dtype=np.uint32)
+        for w in range(M):
+            rows[w, :W] = oracle.pack_bits(s[w])
+        rows[:, W:] = r.integers(0, 2**32, size=(M, ldw - W), dtype=np.uint32)  # garbage in row padding
+        vote = torch.full((W + 4,), CANARY_WORD, dtype=torch.int32, device=DEV)
+        B.majority_vote(torch.from_numpy(rows.view(np.int32)).to(DEV), M, d, ldw, vote)
+        ref = oracle.majority_vote(rows.reshape(-1), M, d, ldw=ldw)
+        got = u32(vote)
+        assert np.array_equal(got[:W], ref), "M=%d d=%d" % (M, d)
+        assert np.all(got[W:] == np.uint32(0xDEADBEEF))
+
+
+def test_majority_vote_ignores_garbage_padding_bits():
+    # padding bits of the last word are the caller's to keep 0; the vote masks them anyway
+    M, d = 3, 40
+    rows = np.full((M, 4), 0xFFFFFFFF, dtype=np.uint32)
+    vote = torch.zeros(4, dtype=torch.int32, device=DEV)
+    B.majority_vote(torch.from_numpy(rows.view(np.int32)).to(DEV), M, d, 4, vote)
+    assert u32(vote)[:2].tolist() == [0xFFFFFFFF, 0xFF]
+
+
+@pytest.mark.parametrize("d", SMALL_D)
+def test_sign_apply_small(d):
+    r = np.random.default_rng(d)
+    W = oracle.words(d)
+    x = np.full(d + 7, CANARY_F, dtype=np.float32)
+    x[:d] = (r.standard_normal(d) * 10.0 ** r.integers(-6, 3, d)).astype(np.float32)
+    vote = oracle.pack_bits(r.integers(0, 2, d, dtype=np.uint8))
+    for delta in (1e-4, 0.37):
+        xd = torch.from_numpy(x).to(DEV)
+        B.sign_apply(xd, torch.from_numpy(vote.view(np.int32)).to(DEV), d, delta)
+        ref = x[:d].copy()
+        oracle.sign_apply(ref, vote, d, delta)
+        got = f32(xd)
+        assert_same_f32(got[:d], ref, "x (d=%d)" % d)
+        assert np.all(got[d:] == np.float32(CANARY_F))
+
+
+@pytest.mark.parametrize("M", SMALL_M)
+def test_whole_step_small(M):
+    for d in (33, 1000, 4097, 70001):
+        for beta, with_m in ((0.9, True), (0.0, True), (0.0, False)):
+            ld, W = wl.round_up(d, 4), oracle.words(d)
+            ldw = wl.round_up(W, 4)
+            g, m, x = rand_inputs(M, d, ld, seed=M * 77 + d)
+            gd, md, xd = (torch.from_numpy(a).to(DEV) for a in (g, m, x))
+            bits = torch.zeros(M, ldw, dtype=torch.int32, device=DEV)
+            vote = torch.zeros(W, dtype=torch.int32, device=DEV)
+            B.signsgd_step(xd, gd, md if with_m else None, M, d, ld, beta, 1e-3, bits, ldw, vote)
+            m_ref, x_ref = m.copy().reshape(-1), x.copy()
+            b_ref, v_ref = oracle.signsgd_step(x_ref, g.reshape(-1), m_ref if with_m else None, M, d,
+                                               beta, 1e-3, ld=ld, ldw=ldw)
+            assert np.array_equal(u32(bits).reshape(-1), b_ref)
+            assert np.array_equal(u32(vote), v_ref)
+            assert_same_f32(f32(xd), x_ref, "x")
+            if with_m:
+                assert_same_f32(f32(md).reshape(-1), m_ref, "m")
+
+
+def test_empty_input_launches_nothing():
+    z = torch.zeros(4, dtype=torch.float32, device=DEV)
+    b = torch.full((4,), CANARY_WORD, dtype=torch.int32, device=DEV)
+    B.sign_pack(z, 1, 0, 0, b, 0)
+    B.signum_momentum_pack(z, z.clone(), 1, 0, 0, 0.9, b, 0)
+    B.majority_vote(b, 1, 0, 0, b.clone())
+    B.sign_apply(z, b, 0, 0.1)
+    B.signsgd_step(z, z.clone(), z.clone(), 1, 0, 0, 0.9, 0.1, b, 0, b.clone())
+    torch.cuda.synchronize()
+    assert np.all(u32(b) == np.uint32(0xDEADBEEF)) and float(z.abs().max()) == 0.0
+
+
+# ------------------------------------------------------------------ the named configurations
+
+def run_config_full(cfg, check_every_step=True):
+    """Run cfg.steps steps on the GPU and in the oracle on identical inputs; compare everything."""
+    M, d, ld, ldw, W = cfg.M, cfg.d, cfg.ld, cfg.ldw, cfg.words
+    shared = cfg.shared(DEV)
+    xd = cfg.x0(DEV)
+    md = cfg.m0(DEV) if cfg.momentum_buffer else None
+    x_ref = f32(xd).copy()
+    m_ref = f32(md).reshape(-1).copy() if md is not None else None
+    bits = torch.zeros(M, ldw, dtype=torch.int32, device=DEV)
+    vote = torch.zeros(W, dtype=torch.int32, device=DEV)
+    for k in range(cfg.steps):
+        gd = cfg.g(k, DEV, shared)
+        B.signsgd_step(xd, gd, md, M, d, ld, cfg.beta, cfg.delta, bits, ldw, vote)
+        g_host = f32(gd).reshape(-1)
+        b_ref, v_ref = oracle.signsgd_step(x_ref, g_host, m_ref, M, d, cfg.beta, cfg.delta, ld=ld, ldw=ldw)
+        if check_every_step or k == cfg.steps - 1:
+            assert np.array_equal(u32(bits).reshape(-1), b_ref), "bits, step %d" % k
+            assert np.array_equal(u32(vote), v_ref), "vote, step %d" % k
+            assert_same_f32(f32(xd), x_ref, "x, step %d" % k)
+            if md is not None:
+                assert_same_f32(f32(md).reshape(-1), m_ref, "m, step %d" % k)
+    return f32(gd), v_ref
+
+
+def test_config1_small_signum_five_steps():
+    run_config_full(wl.small_signum())
+
+
+def test_config2_resnet50_layout():
+    cfg = wl.resnet50_signum()
+    _, v_ref = run_config_full(cfg)
+    # padding elements between tensors hold g = 0, so they vote +1 on both sides
+    votes = oracle.unpack_bits(v_ref, cfg.d)
+    end = cfg.segments[-1][0] + cfg.segments[-1][1]
+    assert end < cfg.d and votes[end:].all()
+
+
+def test_config3_ties_and_zeros():
+    cfg = wl.tie_zero_stress()
+    g, v_ref = run_config_full(cfg)
+    g = g[:, :cfg.d]
+    votes = oracle.unpack_bits(v_ref, cfg.d).astype(bool)
+    P = (~(g < 0)).sum(axis=0)
+    tie = 2 * P == cfg.M
+    assert tie.mean() > 0.30 and votes[tie].all()            # every tie resolves to +1
+    # the same inputs through the fused momentum kernel with beta = 0 give the same words
+    gd = cfg.g(0, DEV)
+    md = torch.randn(cfg.M, cfg.ld, device=DEV)
+    b1 = torch.zeros(cfg.M, cfg.ldw, dtype=torch.int32, device=DEV)
+    b2 = torch.zeros_like(b1)
+    B.sign_pack(gd, cfg.M, cfg.d, cfg.ld, b1, cfg.ldw)
+    B.signum_momentum_pack(gd, md, cfg.M, cfg.d, cfg.ld, 0.0, b2, cfg.ldw)
+    assert torch.equal(b1, b2) and torch.equal(md, gd)
+
+
+def sampled_chunk_parity(cfg, n_chunks, chunk, seed):
+    """Full-size run on the GPU; the oracle recomputes `n_chunks` slices of `chunk` elements from
+    host copies of the very same inputs.  Plus properties that hold at any size, checked in full
+    with plain torch reductions."""
+    M, d, ld, ldw, W = cfg.M, cfg.d, cfg.ld, cfg.ldw, cfg.words
+    shared = cfg.shared(DEV)
+    xd = cfg.x0(DEV)
+    md = cfg.m0(DEV)
+    if cfg.beta > 0:
+        cfg.g(1000, DEV, shared, out=md)                  # a non-trivial starting momentum
+        md.mul_(0.5)
+    gd = cfg.g(0, DEV, shared)
+    r = np.random.default_rng(seed)
+    starts = sorted(set([0, (d - chunk) // 32 * 32] +
+                        [int(o) * 32 for o in r.integers(0, (d - chunk) // 32, n_chunks - 2)]))
+    x0_s = [f32(xd[o:o + chunk]).copy() for o in starts]
+    m0_s = [f32(md[:, o:o + chunk]).copy() for o in starts]
+    bits = torch.zeros(M, ldw, dtype=torch.int32, device=DEV)
+    vote = torch.zeros(W, dtype=torch.int32, device=DEV)
+    x_before_sum = xd.double().sum().item()
+    B.signsgd_step(xd, gd, md, M, d, ld, cfg.beta, cfg.delta, bits, ldw, vote)
+    torch.cuda.synchronize()
+    for o, x_ref, m_ref in zip(starts, x0_s, m0_s):
+        n = min(chunk, d - o)
+        g_s = np.ascontiguousarray(f32(gd[:, o:o + n]))
+        m_flat = np.ascontiguousarray(m_ref).reshape(-1)
+        b_ref, v_ref = oracle.signsgd_step(x_ref, g_s.reshape(-1), m_flat, M, n, cfg.beta, cfg.delta)
+        wn = oracle.words(n)
+        assert np.array_equal(u32(bits[:, o // 32:o // 32 + wn]).reshape(-1), b_ref), "bits @%d" % o
+        assert np.array_equal(u32(vote[o // 32:o // 32 + wn]), v_ref), "vote @%d" % o
+        assert_same_f32(f32(xd[o:o + n]), x_ref, "x @%d" % o)
+        assert_same_f32(f32(md[:, o:o + n]).reshape(-1), m_flat, "m @%d" % o)
+    # any-size properties: popcount of each packed row = number of non-negative momenta;
+    # popcount of the vote tells how far sum(x) moved
+    pops = [int(_popcount(bits[w, :W])) for w in range(M)]
+    nonneg = [int((~(md[w, :d] < 0)).sum().item()) for w in range(M)]
+    assert pops == nonneg
+    pv = int(_popcount(vote))
+    moved = x_before_sum - xd.double().sum().item()
+    assert abs(moved - cfg.delta * (2 * pv - d)) <= 1e-3 * cfg.delta * d + 1e-6
+
+
+def _popcount(t: torch.Tensor) -> int:
+    v = t.to(torch.int64) & 0xFFFFFFFF
+    total = 0
+    for sh in range(0, 32, 8):
+        b = (v >> sh) & 0xFF
+        b = (b & 0x55) + ((b >> 1) & 0x55)
+        b = (b & 0x33) + ((b >> 2) & 0x33)
+        b = (b & 0x0F) + ((b >> 4) & 0x0F)
+        total += int(b.sum().item())
+    return total
+
+
+def test_config4_bert_large_full_size_sampled():
+    free, _ = torch.cuda.mem_get_info()
+    cfg = wl.bert_large_signum()
+    need = 2 * cfg.M * cfg.ld * 4 + 4 * cfg.d * 4 + (8 << 30)
+    if free < need:
+        pytest.skip("needs %.0f GB of free device memory" % (need / 2**30))
+    sampled_chunk_parity(cfg, n_chunks=24, chunk=1 << 20, seed=4)
+
+
+@pytest.mark.parametrize("d,M", [(1 << 10, 31), (1 << 13, 15), (1 << 16, 7), (1 << 20, 3), (1 << 22, 1),
+                                 (1 << 24, 7), (1 << 24, 31)])
+def test_config5_sweep_points_full_parity(d, M):
+    run_config_full(wl.sweep_point(d, M))
+
+
+@pytest.mark.parametrize("d,M", [(1 << 26, 7), (1 << 28, 3)])
+def test_config5_large_sweep_points_sampled(d, M):
+    sampled_chunk_parity(wl.sweep_point(d, M), n_chunks=16, chunk=1 << 20, seed=d % 1000 + M)
+
+
+def test_host_buffer_step_matches_device_step():
+    cfg = wl.small_signum(d=300_001, M=5)
+    M, d, ld, ldw, W = cfg.M, cfg.d, cfg.ld, cfg.ldw, cfg.words
+    g_host = cfg.g(0).pin_memory()
+    x1, x2 = cfg.x0(DEV), cfg.x0(DEV)
+    m1 = torch.randn(M, ld, device=DEV) * 0.1
+    m2 = m1.clone()
+    bits1 = torch.zeros(M, ldw, dtype=torch.int32, device=DEV)
+    bits2, vote1 = torch.zeros_like(bits1), torch.zeros(W, dtype=torch.int32, device=DEV)
+    vote2 = torch.zeros_like(vote1)
+    stage = torch.empty(M, ld, device=DEV)
+    vote_host = torch.zeros(W, dtype=torch.int32).pin_memory()
+    B.signsgd_step(x1, g_host.to(DEV), m1, M, d, ld, cfg.beta, cfg.delta, bits1, ldw, vote1)
+    B.signsgd_step_host(x2, g_host, m2, M, d, ld, cfg.beta, cfg.delta, stage, bits2, ldw, vote2, vote_host)
+    torch.cuda.synchronize()
+    assert torch.equal(x1, x2) and torch.equal(m1, m2) and torch.equal(bits1, bits2)
+    assert torch.equal(vote1.cpu(), vote_host)
+
+
+def test_resume_from_copied_state_is_bit_identical():
+    cfg = wl.small_signum(d=50_000, M=3)
+    M, d, ld, ldw, W = cfg.M, cfg.d, cfg.ld, cfg.ldw, cfg.words
+    mu = cfg.shared(DEV)
+    gs = [cfg.g(k, DEV, mu) for k in range(5)]
+    bits = torch.zeros(M, ldw, dtype=torch.int32, device=DEV)
+    vote = torch.zeros(W, dtype=torch.int32, device=DEV)
+    xa, ma = cfg.x0(DEV), cfg.m0(DEV)
+    for k in range(5):
+        B.signsgd_step(xa, gs[k], ma, M, d, ld, cfg.beta, cfg.delta, bits, ldw, vote)
+    xb, mb = cfg.x0(DEV), cfg.m0(DEV)
+    for k in range(2):
+        B.signsgd_step(xb, gs[k], mb, M, d, ld, cfg.beta, cfg.delta, bits, ldw, vote)
+    xb, mb = xb.cpu().to(DEV), mb.cpu().to(DEV)             # state leaves and re-enters the device
+    for k in range(2, 5):
+        B.signsgd_step(xb, gs[k], mb, M, d, ld, cfg.beta, cfg.delta, bits, ldw, vote)
+    assert torch.equal(xa, xb) and torch.equal(ma, mb)
