@@ -58,7 +58,8 @@ typedef enum {
   SSGD_ERR_ALIGN = 2, /* pointer not 16-byte aligned, or ld / ldw not 4-aligned */
   SSGD_ERR_SIZE = 3,  /* M out of range, ld < d, ldw < W, or a size overflows   */
   SSGD_ERR_ARG = 4,   /* beta outside [0,1) or NaN; delta not finite            */
-  SSGD_ERR_CUDA = 5   /* the CUDA runtime reported an error at launch / copy    */
+  SSGD_ERR_CUDA = 5,  /* the CUDA runtime reported an error at launch / copy    */
+  SSGD_ERR_SCRATCH = 6 /* problem needs more than the library's built-in scratch */
 } ssgd_status;
 
 /* ceil(d / 32): words per packed sign vector (d bits per vector, Table 1). */
@@ -129,6 +130,45 @@ ssgd_status ssgd_signsgd_step_host(float* x, const float* g_host, float* m,
                                    uint32_t* bits_ws, size_t ldw,
                                    uint32_t* vote_ws, uint32_t* vote_host,
                                    void* stream);
+
+/* Capacity, in 32-bit words, of the scratch area that ssgd_signsgd_step_noalloc
+ * uses (16 MiB of device memory per GPU that loads the library, held until the
+ * process exits). */
+#define SSGD_NOALLOC_SCRATCH_WORDS ((size_t)4 << 20)
+
+/* ssgd_signsgd_step for callers that cannot provide the two word workspaces.
+ * (The paper has no counterpart to this call: it is a packaging variant of the
+ * step above, with the same arithmetic and the same results for x and m.)
+ *
+ * Who needs it: code that runs where device memory can no longer be obtained --
+ * for instance an optimiser hook inside a training process whose framework has
+ * already reserved all device memory for its own pool, so that a raw cudaMalloc
+ * would fail, or a latency-sensitive loop that must avoid cudaMalloc / cudaFree
+ * because those calls may synchronise the whole device.  Such a caller owns x,
+ * g and m anyway, but has nowhere to put the packed sign rows and the vote.
+ *
+ * This call takes no workspace arguments and allocates nothing (no cudaMalloc,
+ * cudaFree, or allocating library routine): the M sign rows and the vote live in
+ * a fixed array inside the library, SSGD_NOALLOC_SCRATCH_WORDS words long.  With
+ * W = ssgd_words(d) and W4 = W rounded up to a multiple of 4, the call needs
+ * (M + 1) * W4 words; a larger problem is rejected with SSGD_ERR_SCRATCH before
+ * anything is launched (use ssgd_signsgd_step with your own buffers instead).
+ *
+ *   x in/out [d], g in [M][ld], m in/out [M][ld] (NULL allowed iff beta == 0):
+ *   DEVICE pointers with the same rules as ssgd_signsgd_step.
+ *
+ * The first call on each device looks up the device address of the built-in
+ * array (with that device current) and remembers it; make that first call before
+ * starting any stream capture.  All calls on a device share the one array, and it
+ * keeps whatever the previous call left there; nothing in it has to start at
+ * zero, because every word the step reads back it has written first.  Two calls
+ * whose GPU work can overlap (different streams, or different host threads on the
+ * same device) race on that array: issue them on one stream, or order them
+ * yourself.  The wire words are not returned; callers who want them use
+ * ssgd_signsgd_step. */
+ssgd_status ssgd_signsgd_step_noalloc(float* x, const float* g, float* m,
+                                      size_t M, size_t d, size_t ld, float beta,
+                                      float delta, void* stream);
 
 #ifdef __cplusplus
 }

@@ -50,6 +50,7 @@ def lib() -> ctypes.CDLL:
         "ssgd_sign_apply": [vp, vp, sz, f32, vp],
         "ssgd_signsgd_step": [vp, vp, vp, sz, sz, sz, f32, f32, vp, sz, vp, vp],
         "ssgd_signsgd_step_host": [vp, vp, vp, sz, sz, sz, f32, f32, vp, vp, sz, vp, vp, vp],
+        "ssgd_signsgd_step_noalloc": [vp, vp, vp, sz, sz, sz, f32, f32, vp],
     }
     for name, args in sigs.items():
         fn = getattr(L, name)
@@ -166,3 +167,23 @@ def signsgd_step_host(x: torch.Tensor, g_host: torch.Tensor, m: Optional[torch.T
         _ptr(g_stage, torch.float32, "g_stage"), _ptr(bits_ws, WORD_DTYPE, "bits_ws"), ldw,
         _ptr(vote_ws, WORD_DTYPE, "vote_ws"), _ptr(vote_host, WORD_DTYPE, "vote_host", cuda=False),
         _stream(stream)), "ssgd_signsgd_step_host")
+
+
+NOALLOC_SCRATCH_WORDS = 4 << 20
+
+
+def signsgd_step_noalloc(x: torch.Tensor, g: torch.Tensor, m: Optional[torch.Tensor], M: int, d: int,
+                         ld: int, beta: float, delta: float, stream=None) -> None:
+    """The whole step without workspace arguments, for callers that cannot allocate device memory.
+
+    The packed sign rows and the vote go to a fixed 16 MiB array inside the library, so the problem
+    must satisfy (M + 1) * round_up(ceil(d / 32), 4) <= NOALLOC_SCRATCH_WORDS; larger ones raise
+    (status 6).  Calls on one device share that array: keep them on one stream.  The first call on a
+    device does a one-time address look-up and should come before any stream capture.
+    """
+    _need(x, d, "x"); _need(g, M * ld, "g")
+    if m is not None:
+        _need(m, M * ld, "m")
+    _check(lib().ssgd_signsgd_step_noalloc(
+        _ptr(x, torch.float32, "x"), _ptr(g, torch.float32, "g"), _ptr(m, torch.float32, "m"),
+        M, d, ld, beta, delta, _stream(stream)), "ssgd_signsgd_step_noalloc")

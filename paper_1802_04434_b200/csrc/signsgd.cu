@@ -499,6 +499,7 @@ const char* ssgd_status_str(ssgd_status s) {
     case SSGD_ERR_SIZE: return "worker count out of range, row stride too short, or size overflow";
     case SSGD_ERR_ARG: return "beta outside [0,1) or delta not finite";
     case SSGD_ERR_CUDA: return "CUDA runtime error";
+    case SSGD_ERR_SCRATCH: return "problem exceeds the built-in scratch capacity of the no-allocation call";
   }
   return "unknown status";
 }
@@ -564,3 +565,50 @@ ssgd_status ssgd_signsgd_step_host(float* x, const float* g_host, float* m, size
 }
 
 }  // extern "C"
+
+// ---------------------------------------------------------------------------
+// The step for callers that cannot allocate: its word workspaces live in a fixed
+// array in device memory instead of caller-provided buffers.
+//
+// `noalloc_scratch` below is a device symbol.  Inside host code its name is only
+// a stand-in that the runtime maps to the real array, never a pointer a kernel
+// could use, so the host asks the runtime for the device address once per device
+// and hands that address to the launches.
+
+namespace {
+
+static __device__ __align__(256) uint32_t noalloc_scratch[SSGD_NOALLOC_SCRATCH_WORDS];
+
+constexpr int kMaxDevices = 64;
+uint32_t* noalloc_scratch_addr[kMaxDevices];  // device address per device, filled on first use
+
+// Device address of the scratch array on the current device, or nullptr on error.
+uint32_t* noalloc_scratch_on_current_device() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+  uint32_t* p = __atomic_load_n(&noalloc_scratch_addr[dev], __ATOMIC_ACQUIRE);
+  if (p) return p;
+  void* sym = nullptr;
+  if (cudaGetSymbolAddress(&sym, noalloc_scratch) != cudaSuccess || sym == nullptr) {
+    (void)cudaGetLastError();
+    return nullptr;
+  }
+  p = static_cast<uint32_t*>(sym);
+  __atomic_store_n(&noalloc_scratch_addr[dev], p, __ATOMIC_RELEASE);  // same value from any thread
+  return p;
+}
+
+}  // namespace
+
+extern "C" ssgd_status ssgd_signsgd_step_noalloc(float* x, const float* g, float* m, size_t M,
+                                                 size_t d, size_t ld, float beta, float delta,
+                                                 void* stream) {
+  if (M < 1 || M > SSGD_MAX_WORKERS || d > SIZE_MAX - 127) return SSGD_ERR_SIZE;
+  const size_t W4 = (ssgd_words(d) + 3) / 4 * 4;              // row stride: keeps rows 16-byte aligned
+  if (W4 > SSGD_NOALLOC_SCRATCH_WORDS / (M + 1)) return SSGD_ERR_SCRATCH;
+  uint32_t* scratch = noalloc_scratch_on_current_device();
+  if (!scratch) return SSGD_ERR_CUDA;
+  uint32_t* bits_ws = scratch;                                 // [M][W4]
+  uint32_t* vote_ws = scratch + M * W4;                        // [W4]
+  return ssgd_signsgd_step(x, g, m, M, d, ld, beta, delta, bits_ws, W4, vote_ws, stream);
+}
