@@ -22,22 +22,39 @@ namespace {
 // ---------------------------------------------------------------------------
 // small device helpers
 
-// Streaming 128-bit accesses: the data is touched once, so it should neither
-// stay in L1 nor displace useful lines in L2.
-__device__ __forceinline__ float4 ld_stream(const float* p) {
-  return __ldcs(reinterpret_cast<const float4*>(p));
+// 128-bit accesses.  Loads use the default caching path and stores the streaming
+// one: measured on B200 this pair, with one tile per CTA, streams faster than a
+// device-to-device copy, while evict-first loads and persistent grids were 8-10 %
+// slower.
+__device__ __forceinline__ float4 ld128(const float* p) {
+  return *reinterpret_cast<const float4*>(p);
 }
-__device__ __forceinline__ void st_stream(float* p, float4 v) {
+__device__ __forceinline__ void st128(float* p, float4 v) {
   __stcs(reinterpret_cast<float4*>(p), v);
 }
 
 // sign(.) of Algorithms 1-3 in one bit: +0, -0 and NaN all count as +1.
 __device__ __forceinline__ unsigned sign_bit(float v) { return (v < 0.0f) ? 0u : 1u; }
 
+__device__ __forceinline__ unsigned sign_nibble(const float4& v) {
+  return sign_bit(v.x) | (sign_bit(v.y) << 1) | (sign_bit(v.z) << 2) | (sign_bit(v.w) << 3);
+}
+
 // Algorithm 2, second step, as two correctly rounded fp32 operations.  Written
 // with explicit intrinsics so that the compiler can neither contract nor split them.
 __device__ __forceinline__ float momentum_update(float beta, float omb, float m, float g) {
   return __fmaf_rn(beta, m, __fmul_rn(omb, g));
+}
+__device__ __forceinline__ float4 momentum_update4(float beta, float omb, const float4& m, const float4& g) {
+  return make_float4(momentum_update(beta, omb, m.x, g.x), momentum_update(beta, omb, m.y, g.y),
+                     momentum_update(beta, omb, m.z, g.z), momentum_update(beta, omb, m.w, g.w));
+}
+
+// Algorithm 3, worker block: four parameters move by -delta or +delta according
+// to four voted bits (bit set = sign +1 = subtract delta).
+__device__ __forceinline__ float4 apply4(const float4& x, unsigned nib, float delta, float minus) {
+  return make_float4(__fadd_rn(x.x, (nib & 1u) ? minus : delta), __fadd_rn(x.y, (nib & 2u) ? minus : delta),
+                     __fadd_rn(x.z, (nib & 4u) ? minus : delta), __fadd_rn(x.w, (nib & 8u) ? minus : delta));
 }
 
 // A warp holds 128 consecutive elements, lane l the four elements 4l..4l+3.
@@ -49,25 +66,35 @@ __device__ __forceinline__ unsigned assemble_word(unsigned nibble, unsigned lane
   return __reduce_or_sync(group_mask, nibble << (4u * (lane & 7u)));
 }
 
-// ---------------------------------------------------------------------------
-// worker kernel: [momentum update +] sign + 1-bit pack, all M rows in one launch
-//
-// Work is cut into tiles of TILE = THREADS * 4 * UNROLL elements of one row.  A
-// warp owns 128 * UNROLL consecutive elements of the tile, so that the words it
-// produces are consecutive too.  Tiles are numbered row-major over (row, tile in
-// row) and dealt to CTAs round-robin.
+// Tiling shared by the worker, apply and fused kernels: a CTA of kThreads threads
+// owns a tile of kThreads * 4 * UNROLL consecutive elements of one row, a warp
+// 128 * UNROLL consecutive elements of it ("span"), so that a warp's words are
+// consecutive too: its span covers words (e0 / 32) + 4u + j for unroll step u and
+// lane group j = lane / 8.
+constexpr int kThreads = 256;
 
-constexpr int kWorkerThreads = 256;
+// Within a group of eight lanes all lanes hold the same assembled word.  Lane
+// (lane % 8) == u keeps the word of unroll step u ("its" word), so that after the
+// UNROLL steps the 4 * UNROLL words of the span sit in 4 * UNROLL distinct lanes
+// and can be stored, or counted, once each.
+template <int UNROLL>
+__device__ __forceinline__ unsigned long long own_word_index(unsigned lane) {
+  return (unsigned long long)(lane & 7u) * 4u + (lane >> 3);   // valid for lane % 8 < UNROLL
+}
+
+// ---------------------------------------------------------------------------
+// worker kernel: [momentum update +] sign + 1-bit pack, all M rows in one launch.
+// Tiles are numbered row-major over (row, tile in row), one tile per CTA.
 
 template <bool MOMENTUM, int UNROLL>
-__global__ void __launch_bounds__(kWorkerThreads)
+__global__ void __launch_bounds__(kThreads)
 worker_pack_kernel(const float* __restrict__ g, float* __restrict__ m,
                    uint32_t* __restrict__ bits, unsigned long long d,
                    unsigned long long ld, unsigned long long ldw,
                    unsigned long long tiles_per_row, unsigned long long total_tiles,
                    float beta, float omb) {
-  constexpr unsigned long long TILE = (unsigned long long)kWorkerThreads * 4 * UNROLL;
-  constexpr unsigned WARP_SPAN = 128 * UNROLL;
+  constexpr unsigned long long TILE = (unsigned long long)kThreads * 4 * UNROLL;
+  constexpr unsigned SPAN = 128 * UNROLL;
   const unsigned lane = threadIdx.x & 31u;
   const unsigned warp = threadIdx.x >> 5;
 
@@ -75,36 +102,33 @@ worker_pack_kernel(const float* __restrict__ g, float* __restrict__ m,
     const unsigned long long row = t / tiles_per_row;
     const unsigned long long tile = t - row * tiles_per_row;
     // first element of this warp's span, within the row
-    const unsigned long long e0 = tile * TILE + (unsigned long long)warp * WARP_SPAN;
+    const unsigned long long e0 = tile * TILE + (unsigned long long)warp * SPAN;
     if (e0 >= d) continue;
     const float* gr = g + row * ld;
     float* mr = MOMENTUM ? m + row * ld : nullptr;
     uint32_t* br = bits + row * ldw + (e0 >> 5);
+    unsigned mine = 0;
 
-    if (e0 + WARP_SPAN <= d) {
+    if (e0 + SPAN <= d) {
       // interior: no bounds checks, all loads issued before any use
       float4 gv[UNROLL], mv[UNROLL];
 #pragma unroll
-      for (int u = 0; u < UNROLL; ++u) gv[u] = ld_stream(gr + e0 + u * 128 + lane * 4);
+      for (int u = 0; u < UNROLL; ++u) gv[u] = ld128(gr + e0 + u * 128 + lane * 4);
       if (MOMENTUM) {
 #pragma unroll
-        for (int u = 0; u < UNROLL; ++u) mv[u] = ld_stream(mr + e0 + u * 128 + lane * 4);
+        for (int u = 0; u < UNROLL; ++u) mv[u] = ld128(mr + e0 + u * 128 + lane * 4);
       }
 #pragma unroll
       for (int u = 0; u < UNROLL; ++u) {
         float4 v = gv[u];
         if (MOMENTUM) {
-          v.x = momentum_update(beta, omb, mv[u].x, v.x);
-          v.y = momentum_update(beta, omb, mv[u].y, v.y);
-          v.z = momentum_update(beta, omb, mv[u].z, v.z);
-          v.w = momentum_update(beta, omb, mv[u].w, v.w);
-          st_stream(mr + e0 + u * 128 + lane * 4, v);
+          v = momentum_update4(beta, omb, mv[u], v);
+          st128(mr + e0 + u * 128 + lane * 4, v);
         }
-        const unsigned nib = sign_bit(v.x) | (sign_bit(v.y) << 1) | (sign_bit(v.z) << 2) |
-                             (sign_bit(v.w) << 3);
-        const unsigned word = assemble_word(nib, lane);
-        if ((lane & 7u) == 0) br[u * 4 + (lane >> 3)] = word;
+        const unsigned word = assemble_word(sign_nibble(v), lane);
+        if ((lane & 7u) == (unsigned)u) mine = word;
       }
+      if ((lane & 7u) < (unsigned)UNROLL) br[own_word_index<UNROLL>(lane)] = mine;
     } else {
       // ragged end of the row: element-wise guards, padding bits stay 0, and
       // nothing at or beyond d is written
@@ -134,11 +158,10 @@ worker_pack_kernel(const float* __restrict__ g, float* __restrict__ m,
 // ---------------------------------------------------------------------------
 // majority vote: bit-sliced vertical counter
 //
-// One thread owns four consecutive words (128 parameters) and walks down the M
-// rows.  The count of set bits per parameter is kept as NP bit-planes (plane p
-// holds bit p of all 128 counters), and rows are folded in with carry-save
-// adders (3 words in, sum + carry out: one XOR3 and one MAJ3 per word), eight
-// rows per block, so the cost is about two logic operations per input word.
+// The count of set bits per parameter is kept as NP bit-planes (plane p holds
+// bit p of 32 counters per word), and rows are folded in with carry-save adders
+// (3 words in, sum + carry out: one XOR3 and one MAJ3 per word), eight rows per
+// block, so the cost is about two logic operations per input word.
 //
 // The comparison with the threshold T = ceil(M/2) is folded into the counter's
 // start value: with L = NP - 1 chosen so that floor(M/2) < 2^L, the counter
@@ -149,7 +172,7 @@ struct W4 {
   unsigned x, y, z, w;
 };
 __device__ __forceinline__ W4 ld_words(const uint32_t* p) {
-  const uint4 v = __ldcs(reinterpret_cast<const uint4*>(p));
+  const uint4 v = *reinterpret_cast<const uint4*>(p);
   return W4{v.x, v.y, v.z, v.w};
 }
 __device__ __forceinline__ unsigned xor3(unsigned a, unsigned b, unsigned c) { return a ^ b ^ c; }
@@ -204,16 +227,45 @@ struct Counter {
   }
 };
 
-constexpr int kVoteThreads = 256;
-
+// The same counter on a single word per thread (used by the fused step kernel).
 template <int NP>
-__global__ void __launch_bounds__(kVoteThreads)
+struct Counter1 {
+  unsigned c[NP];
+  __device__ __forceinline__ void init(unsigned start_value) {
+#pragma unroll
+    for (int p = 0; p < NP; ++p) c[p] = ((start_value >> p) & 1u) ? 0xFFFFFFFFu : 0u;
+  }
+  template <int K>
+  __device__ __forceinline__ void add(unsigned v) {
+#pragma unroll
+    for (int p = K; p < NP; ++p) {
+      const unsigned carry = c[p] & v;
+      c[p] ^= v;
+      v = carry;
+    }
+  }
+  __device__ __forceinline__ void add2(unsigned a, unsigned b) {
+    if (NP >= 2) {
+      const unsigned h = maj3(c[0], a, b);
+      c[0] = xor3(c[0], a, b);
+      add<1>(h);
+    } else {
+      add<0>(a);   // not reached: one plane means one row
+    }
+  }
+  __device__ __forceinline__ unsigned top() const { return c[NP - 1]; }
+};
+
+// One thread owns four consecutive words (one 128-bit load per row) and walks
+// down the M rows; one 256-thread CTA covers 1024 words.
+template <int NP>
+__global__ void __launch_bounds__(kThreads)
 vote_kernel(const uint32_t* __restrict__ bits, unsigned M, unsigned long long d,
             unsigned long long W, unsigned long long ldw, uint32_t* __restrict__ vote,
             unsigned start_value) {
   const unsigned long long chunks = (W + 3) / 4;
-  const unsigned long long stride = (unsigned long long)gridDim.x * kVoteThreads;
-  for (unsigned long long q = (unsigned long long)blockIdx.x * kVoteThreads + threadIdx.x;
+  const unsigned long long stride = (unsigned long long)gridDim.x * kThreads;
+  for (unsigned long long q = (unsigned long long)blockIdx.x * kThreads + threadIdx.x;
        q < chunks; q += stride) {
     const uint32_t* col = bits + 4 * q;
     Counter<NP> cnt;
@@ -270,42 +322,33 @@ vote_kernel(const uint32_t* __restrict__ bits, unsigned M, unsigned long long d,
 
 // ---------------------------------------------------------------------------
 // apply: x <- x -/+ delta by the voted bit.  Thread layout as in the worker
-// kernel: lane l of a warp holds elements 4l..4l+3 of a 128-element span, whose
-// four bits sit at position 4(l%8) of word l/8 of the span.
-
-constexpr int kApplyThreads = 256;
+// kernel: lane l of a warp holds elements 4l..4l+3 of a 128-element step, whose
+// four bits sit at position 4(l%8) of word l/8 of that step.
 
 template <int UNROLL>
-__global__ void __launch_bounds__(kApplyThreads)
+__global__ void __launch_bounds__(kThreads)
 apply_kernel(float* __restrict__ x, const uint32_t* __restrict__ vote, unsigned long long d,
              unsigned long long total_tiles, float delta) {
-  constexpr unsigned long long TILE = (unsigned long long)kApplyThreads * 4 * UNROLL;
-  constexpr unsigned WARP_SPAN = 128 * UNROLL;
+  constexpr unsigned long long TILE = (unsigned long long)kThreads * 4 * UNROLL;
+  constexpr unsigned SPAN = 128 * UNROLL;
   const unsigned lane = threadIdx.x & 31u;
   const unsigned warp = threadIdx.x >> 5;
   const float minus = -delta;
   for (unsigned long long t = blockIdx.x; t < total_tiles; t += gridDim.x) {
-    const unsigned long long e0 = t * TILE + (unsigned long long)warp * WARP_SPAN;
+    const unsigned long long e0 = t * TILE + (unsigned long long)warp * SPAN;
     if (e0 >= d) continue;
     const uint32_t* vw = vote + (e0 >> 5);
-    if (e0 + WARP_SPAN <= d) {
+    if (e0 + SPAN <= d) {
       float4 xv[UNROLL];
       unsigned wv[UNROLL];
 #pragma unroll
       for (int u = 0; u < UNROLL; ++u) {
-        xv[u] = ld_stream(x + e0 + u * 128 + lane * 4);
+        xv[u] = ld128(x + e0 + u * 128 + lane * 4);
         wv[u] = __ldg(vw + u * 4 + (lane >> 3));
       }
 #pragma unroll
-      for (int u = 0; u < UNROLL; ++u) {
-        const unsigned nib = wv[u] >> (4u * (lane & 7u));
-        float4 v = xv[u];
-        v.x = __fadd_rn(v.x, (nib & 1u) ? minus : delta);
-        v.y = __fadd_rn(v.y, (nib & 2u) ? minus : delta);
-        v.z = __fadd_rn(v.z, (nib & 4u) ? minus : delta);
-        v.w = __fadd_rn(v.w, (nib & 8u) ? minus : delta);
-        st_stream(x + e0 + u * 128 + lane * 4, v);
-      }
+      for (int u = 0; u < UNROLL; ++u)
+        st128(x + e0 + u * 128 + lane * 4, apply4(xv[u], wv[u] >> (4u * (lane & 7u)), delta, minus));
     } else {
 #pragma unroll 1
       for (int u = 0; u < UNROLL; ++u) {
@@ -317,6 +360,120 @@ apply_kernel(float* __restrict__ x, const uint32_t* __restrict__ vote, unsigned 
             x[e + k] = __fadd_rn(x[e + k], bit ? minus : delta);
           }
         }
+      }
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------
+// fused step: one launch does the worker step for all M rows, the vote and the
+// apply on a tile of columns, so that the sign words are never read back from
+// memory and x is touched by the CTA that voted on it.  Per parameter it moves
+// 12.125 M + 8.125 bytes (g and m of every row, the M sign words and the vote
+// word written out as the wire data, x read and written).
+//
+// A CTA owns columns [tile * TILE, (tile + 1) * TILE) and walks the M rows.  For
+// every row each warp does what the worker kernel does on its span; the lane
+// that keeps "its" word (see own_word_index) stores it to the row's sign words
+// and folds it into a private bit-sliced counter.  After the last row the top
+// plane of that counter is the voted word; it is stored and handed back to the
+// eight lanes of its group by shuffles for the update of x.
+
+template <bool MOMENTUM, int UNROLL, int NP>
+__global__ void __launch_bounds__(kThreads)
+fused_step_kernel(const float* __restrict__ g, float* __restrict__ m, float* __restrict__ x,
+                  uint32_t* __restrict__ bits, uint32_t* __restrict__ vote, unsigned M,
+                  unsigned long long d, unsigned long long ld, unsigned long long ldw,
+                  float beta, float omb, float delta, unsigned start_value) {
+  constexpr unsigned long long TILE = (unsigned long long)kThreads * 4 * UNROLL;
+  constexpr unsigned SPAN = 128 * UNROLL;
+  const unsigned lane = threadIdx.x & 31u;
+  const unsigned warp = threadIdx.x >> 5;
+  const unsigned sub = lane & 7u;
+  const float minus = -delta;
+  const unsigned long long e0 = (unsigned long long)blockIdx.x * TILE + (unsigned long long)warp * SPAN;
+  if (e0 >= d) return;   // uniform over the warp; nothing below synchronises across warps
+
+  Counter1<NP> cnt;
+  cnt.init(start_value);
+  const unsigned long long w0 = e0 >> 5;                      // first word of the span
+  const unsigned long long my_word = w0 + own_word_index<UNROLL>(lane);
+
+  if (e0 + SPAN <= d) {
+    const unsigned long long off = e0 + lane * 4;
+    for (unsigned row = 0; row < M; ++row) {
+      const float* gr = g + (unsigned long long)row * ld + off;
+      float* mr = MOMENTUM ? m + (unsigned long long)row * ld + off : nullptr;
+      float4 gv[UNROLL], mv[UNROLL];
+#pragma unroll
+      for (int u = 0; u < UNROLL; ++u) gv[u] = ld128(gr + u * 128);
+      if (MOMENTUM) {
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) mv[u] = ld128(mr + u * 128);
+      }
+      unsigned mine = 0;
+#pragma unroll
+      for (int u = 0; u < UNROLL; ++u) {
+        float4 v = gv[u];
+        if (MOMENTUM) {
+          v = momentum_update4(beta, omb, mv[u], v);
+          st128(mr + u * 128, v);
+        }
+        const unsigned word = assemble_word(sign_nibble(v), lane);
+        if (sub == (unsigned)u) mine = word;
+      }
+      if (sub < (unsigned)UNROLL) bits[(unsigned long long)row * ldw + my_word] = mine;
+      cnt.template add<0>(mine);
+    }
+    const unsigned voted = cnt.top();
+    if (sub < (unsigned)UNROLL) vote[my_word] = voted;
+    float4 xv[UNROLL];
+#pragma unroll
+    for (int u = 0; u < UNROLL; ++u) xv[u] = ld128(x + off + u * 128);
+#pragma unroll
+    for (int u = 0; u < UNROLL; ++u) {
+      const unsigned vw = __shfl_sync(0xFFFFFFFFu, voted, (lane & 24u) + u);  // owner of step u in my group
+      st128(x + off + u * 128, apply4(xv[u], vw >> (4u * sub), delta, minus));
+    }
+  } else {
+    // ragged end of the vector: the same walk with element-wise guards.  Bits at
+    // positions >= d stay 0 in every row, so they count 0 votes and the voted
+    // word has them 0 as well (the threshold is at least 1).
+    for (unsigned row = 0; row < M; ++row) {
+      const float* gr = g + (unsigned long long)row * ld;
+      float* mr = MOMENTUM ? m + (unsigned long long)row * ld : nullptr;
+      unsigned mine = 0;
+#pragma unroll 1
+      for (int u = 0; u < UNROLL; ++u) {
+        const unsigned long long e = e0 + u * 128 + lane * 4;
+        unsigned nib = 0;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          if (e + k < d) {
+            float v = gr[e + k];
+            if (MOMENTUM) {
+              v = momentum_update(beta, omb, mr[e + k], v);
+              mr[e + k] = v;
+            }
+            nib |= sign_bit(v) << k;
+          }
+        }
+        const unsigned word = assemble_word(nib, lane);
+        if (sub == (unsigned)u) mine = word;
+      }
+      // my word exists iff its first element is below d
+      if (sub < (unsigned)UNROLL && my_word * 32 < d) bits[(unsigned long long)row * ldw + my_word] = mine;
+      cnt.template add<0>(mine);
+    }
+    const unsigned voted = cnt.top();
+    if (sub < (unsigned)UNROLL && my_word * 32 < d) vote[my_word] = voted;
+#pragma unroll 1
+    for (int u = 0; u < UNROLL; ++u) {
+      const unsigned vw = __shfl_sync(0xFFFFFFFFu, voted, (lane & 24u) + u);
+      const unsigned long long e = e0 + u * 128 + lane * 4;
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        if (e + k < d) x[e + k] = __fadd_rn(x[e + k], ((vw >> (4u * sub + k)) & 1u) ? minus : delta);
       }
     }
   }
@@ -365,12 +522,31 @@ inline bool beta_ok(float beta) { return beta >= 0.0f && beta < 1.0f; }  // fals
 
 ssgd_status launch_status() { return cudaGetLastError() == cudaSuccess ? SSGD_OK : SSGD_ERR_CUDA; }
 
-constexpr int kWorkerUnroll = 4;
-constexpr int kApplyUnroll = 4;
+// One tile per CTA; the kernels keep a grid-stride loop for grids beyond the limit.
+constexpr unsigned long long kMaxGrid = 0x7FFFFFFFull;
+unsigned grid_for(unsigned long long ctas) { return (unsigned)(ctas < kMaxGrid ? ctas : kMaxGrid); }
 
-unsigned grid_for(unsigned long long work_items, int sms, int ctas_per_sm) {
-  const unsigned long long full = (unsigned long long)sms * ctas_per_sm;
-  return (unsigned)(work_items < full ? work_items : full);
+// Elements per thread: 4 * unroll.  Large inputs take unroll 4 (eight 128-bit
+// loads in flight per thread in the worker step); smaller ones shrink the tile so
+// that the launch still fills the machine with a few CTAs per SM.
+int pick_unroll(unsigned long long elements_per_row, unsigned long long rows, int sms) {
+  const unsigned long long want = 8ull * sms;                  // CTAs
+  for (int u = 4; u > 1; u /= 2) {
+    const unsigned long long tile = (unsigned long long)kThreads * 4 * u;
+    if (((elements_per_row + tile - 1) / tile) * rows >= want) return u;
+  }
+  return 1;
+}
+
+template <bool MOMENTUM, int UNROLL>
+void launch_worker_u(const float* g, float* m, size_t M, size_t d, size_t ld, float beta,
+                     uint32_t* bits, size_t ldw, cudaStream_t s) {
+  constexpr unsigned long long TILE = (unsigned long long)kThreads * 4 * UNROLL;
+  const unsigned long long tiles_per_row = (d + TILE - 1) / TILE;
+  const unsigned long long total = tiles_per_row * M;
+  const float omb = 1.0f - beta;
+  worker_pack_kernel<MOMENTUM, UNROLL><<<grid_for(total), kThreads, 0, s>>>(
+      g, m, bits, d, ld, ldw, tiles_per_row, total, beta, omb);
 }
 
 template <bool MOMENTUM>
@@ -378,13 +554,11 @@ ssgd_status launch_worker(const float* g, float* m, size_t M, size_t d, size_t l
                           uint32_t* bits, size_t ldw, cudaStream_t s) {
   DeviceInfo di;
   if (!device_info(&di)) return SSGD_ERR_CUDA;
-  constexpr unsigned long long TILE = (unsigned long long)kWorkerThreads * 4 * kWorkerUnroll;
-  const unsigned long long tiles_per_row = (d + TILE - 1) / TILE;
-  const unsigned long long total = tiles_per_row * M;
-  const unsigned grid = grid_for(total, di.sms, 8);
-  const float omb = 1.0f - beta;
-  worker_pack_kernel<MOMENTUM, kWorkerUnroll><<<grid, kWorkerThreads, 0, s>>>(
-      g, m, bits, d, ld, ldw, tiles_per_row, total, beta, omb);
+  switch (pick_unroll(d, M, di.sms)) {
+    case 4: launch_worker_u<MOMENTUM, 4>(g, m, M, d, ld, beta, bits, ldw, s); break;
+    case 2: launch_worker_u<MOMENTUM, 2>(g, m, M, d, ld, beta, bits, ldw, s); break;
+    default: launch_worker_u<MOMENTUM, 1>(g, m, M, d, ld, beta, bits, ldw, s); break;
+  }
   return launch_status();
 }
 
@@ -394,22 +568,22 @@ unsigned vote_planes(size_t M) {
   return L + 1;
 }
 
+// counter start value 2^(NP-1) - ceil(M/2), see the vote kernel
+unsigned vote_start_value(size_t M, unsigned planes) {
+  return (1u << (planes - 1)) - (unsigned)((M + 1) / 2);
+}
+
 template <int NP>
 void launch_vote_np(const uint32_t* bits, size_t M, size_t d, size_t W, size_t ldw, uint32_t* vote,
                     unsigned grid, cudaStream_t s) {
-  const unsigned T = (unsigned)((M + 1) / 2);
-  const unsigned start = (1u << (NP - 1)) - T;
-  vote_kernel<NP><<<grid, kVoteThreads, 0, s>>>(bits, (unsigned)M, d, W, ldw, vote, start);
+  vote_kernel<NP><<<grid, kThreads, 0, s>>>(bits, (unsigned)M, d, W, ldw, vote, vote_start_value(M, NP));
 }
 
 ssgd_status launch_vote(const uint32_t* bits, size_t M, size_t d, size_t ldw, uint32_t* vote,
                         cudaStream_t s) {
-  DeviceInfo di;
-  if (!device_info(&di)) return SSGD_ERR_CUDA;
   const size_t W = ssgd_words(d);
   const unsigned long long chunks = (W + 3) / 4;
-  const unsigned long long ctas = (chunks + kVoteThreads - 1) / kVoteThreads;
-  const unsigned grid = grid_for(ctas, di.sms, 8);
+  const unsigned grid = grid_for((chunks + kThreads - 1) / kThreads);
   switch (vote_planes(M)) {
     case 1: launch_vote_np<1>(bits, M, d, W, ldw, vote, grid, s); break;
     case 2: launch_vote_np<2>(bits, M, d, W, ldw, vote, grid, s); break;
@@ -427,13 +601,79 @@ ssgd_status launch_vote(const uint32_t* bits, size_t M, size_t d, size_t ldw, ui
   return launch_status();
 }
 
+template <int UNROLL>
+void launch_apply_u(float* x, const uint32_t* vote, size_t d, float delta, cudaStream_t s) {
+  constexpr unsigned long long TILE = (unsigned long long)kThreads * 4 * UNROLL;
+  const unsigned long long total = (d + TILE - 1) / TILE;
+  apply_kernel<UNROLL><<<grid_for(total), kThreads, 0, s>>>(x, vote, d, total, delta);
+}
+
 ssgd_status launch_apply(float* x, const uint32_t* vote, size_t d, float delta, cudaStream_t s) {
   DeviceInfo di;
   if (!device_info(&di)) return SSGD_ERR_CUDA;
-  constexpr unsigned long long TILE = (unsigned long long)kApplyThreads * 4 * kApplyUnroll;
-  const unsigned long long total = (d + TILE - 1) / TILE;
-  const unsigned grid = grid_for(total, di.sms, 8);
-  apply_kernel<kApplyUnroll><<<grid, kApplyThreads, 0, s>>>(x, vote, d, total, delta);
+  switch (pick_unroll(d, 1, di.sms)) {
+    case 4: launch_apply_u<4>(x, vote, d, delta, s); break;
+    case 2: launch_apply_u<2>(x, vote, d, delta, s); break;
+    default: launch_apply_u<1>(x, vote, d, delta, s); break;
+  }
+  return launch_status();
+}
+
+struct StepArgs {
+  const float* g;
+  float* m;
+  float* x;
+  uint32_t* bits;
+  uint32_t* vote;
+  size_t M, d, ld, ldw;
+  float beta, delta;
+};
+
+template <bool MOMENTUM, int UNROLL, int NP>
+void launch_fused_mun(const StepArgs& a, cudaStream_t s) {
+  constexpr unsigned long long TILE = (unsigned long long)kThreads * 4 * UNROLL;
+  const unsigned long long tiles = (a.d + TILE - 1) / TILE;
+  fused_step_kernel<MOMENTUM, UNROLL, NP><<<(unsigned)tiles, kThreads, 0, s>>>(
+      a.g, a.m, a.x, a.bits, a.vote, (unsigned)a.M, a.d, a.ld, a.ldw, a.beta, 1.0f - a.beta, a.delta,
+      vote_start_value(a.M, NP));
+}
+
+template <bool MOMENTUM, int UNROLL>
+bool launch_fused_mu(const StepArgs& a, cudaStream_t s) {
+  switch (vote_planes(a.M)) {
+    case 1: launch_fused_mun<MOMENTUM, UNROLL, 1>(a, s); return true;
+    case 2: launch_fused_mun<MOMENTUM, UNROLL, 2>(a, s); return true;
+    case 3: launch_fused_mun<MOMENTUM, UNROLL, 3>(a, s); return true;
+    case 4: launch_fused_mun<MOMENTUM, UNROLL, 4>(a, s); return true;
+    case 5: launch_fused_mun<MOMENTUM, UNROLL, 5>(a, s); return true;
+    case 6: launch_fused_mun<MOMENTUM, UNROLL, 6>(a, s); return true;
+    case 7: launch_fused_mun<MOMENTUM, UNROLL, 7>(a, s); return true;
+    case 8: launch_fused_mun<MOMENTUM, UNROLL, 8>(a, s); return true;
+    case 9: launch_fused_mun<MOMENTUM, UNROLL, 9>(a, s); return true;
+    case 10: launch_fused_mun<MOMENTUM, UNROLL, 10>(a, s); return true;
+    case 11: launch_fused_mun<MOMENTUM, UNROLL, 11>(a, s); return true;
+  }
+  return false;
+}
+
+// The fused kernel's grid is one CTA per tile of columns; vectors too long for
+// one grid (beyond 2^31 tiles) take the three-kernel path instead.
+template <bool MOMENTUM>
+ssgd_status launch_fused(const StepArgs& a, cudaStream_t s, bool* launched) {
+  DeviceInfo di;
+  if (!device_info(&di)) return SSGD_ERR_CUDA;
+  const int unroll = pick_unroll(a.d, 1, di.sms);
+  const unsigned long long tile = (unsigned long long)kThreads * 4 * unroll;
+  *launched = false;
+  if ((a.d + tile - 1) / tile > kMaxGrid) return SSGD_OK;
+  bool ok;
+  switch (unroll) {
+    case 4: ok = launch_fused_mu<MOMENTUM, 4>(a, s); break;
+    case 2: ok = launch_fused_mu<MOMENTUM, 2>(a, s); break;
+    default: ok = launch_fused_mu<MOMENTUM, 1>(a, s); break;
+  }
+  if (!ok) return SSGD_ERR_SIZE;
+  *launched = true;
   return launch_status();
 }
 
@@ -537,6 +777,11 @@ ssgd_status ssgd_signsgd_step(float* x, const float* g, float* m, size_t M, size
   ssgd_status st = check_step(x, g, m, M, d, ld, beta, delta, bits_ws, ldw, vote_ws);
   if (st != SSGD_OK || d == 0) return st;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const StepArgs a{g, m, x, bits_ws, vote_ws, M, d, ld, ldw, beta, delta};
+  bool launched = false;
+  st = m ? launch_fused<true>(a, s, &launched) : launch_fused<false>(a, s, &launched);
+  if (st != SSGD_OK || launched) return st;
+  // vectors beyond one grid of tiles: the same step as three launches
   st = m ? launch_worker<true>(g, m, M, d, ld, beta, bits_ws, ldw, s)
          : launch_worker<false>(g, nullptr, M, d, ld, 0.0f, bits_ws, ldw, s);
   if (st != SSGD_OK) return st;

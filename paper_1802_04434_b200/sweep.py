@@ -1,0 +1,132 @@
+"""Per-kernel bandwidth sweep: d = 2^10 .. 2^28, M in {1, 3, 7, 15, 31}, Signum beta = 0.9.
+
+    python -m paper_1802_04434_b200.sweep [--min-log2 10] [--max-log2 28] [--workers 1,3,7,15,31]
+                                          [--reps 20] [--out sweep.tsv]
+
+For every point and every kernel of the step (worker momentum + pack, majority vote, apply) and for
+the whole step, prints the time per launch, the algorithmic GB/s and its fraction of the measured
+copy peak.  Launches are replayed from a CUDA graph between two CUDA events.  When
+one launch touches less than twice the L2 size, the launches rotate over several buffer sets so that
+the combined footprint exceeds it (column `cold` = 1); for the smallest sizes that would need more
+sets than are allowed and the figures are launch-latency numbers, not bandwidth (cold = 0).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+
+import torch
+
+from . import binding as B
+
+L2_BYTES = 126 << 20
+MAX_SETS = 48
+
+
+def peak_gbs() -> float:
+    p = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "MEASURED_PEAKS.json")
+    try:
+        with open(p) as fh:
+            return float(json.load(fh)["hbm_gbs"])
+    except Exception:
+        return 6650.0
+
+
+def time_launches(fn, n_sets: int, reps: int) -> float:
+    """Average milliseconds per launch of fn(set_index).
+
+    The launches are captured once into a CUDA graph (at least 32 per replay, cycling over the
+    buffer sets) and the graph is replayed `reps` times between two events, so that the host's
+    per-call cost does not limit short kernels."""
+    for s in range(n_sets):
+        fn(s)
+    torch.cuda.synchronize()
+    inner = max(1, -(-32 // n_sets))
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        for _ in range(inner):
+            for s in range(n_sets):
+                fn(s)
+    graph.replay()
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in range(reps):
+        graph.replay()
+    b.record()
+    torch.cuda.synchronize()
+    return a.elapsed_time(b) / (reps * inner * n_sets)
+
+
+def run_point(d: int, M: int, reps: int, dev) -> list:
+    ld = (d + 3) // 4 * 4
+    W = (d + 31) // 32
+    ldw = (W + 3) // 4 * 4
+    beta, delta = 0.9, 1e-4
+    bytes_worker = 12.125 * M * d
+    bytes_vote = (M + 1) / 8.0 * d
+    bytes_apply = 8.125 * d
+    n_sets = int(min(MAX_SETS, max(1, -(-2 * L2_BYTES // int(bytes_vote + 1)))))
+    n_sets_big = int(min(MAX_SETS, max(1, -(-2 * L2_BYTES // int(bytes_worker + 1)))))
+    g = [torch.randn(M, ld, device=dev) for _ in range(n_sets_big)]
+    m = [torch.zeros(M, ld, device=dev) for _ in range(n_sets_big)]
+    n_x = int(min(MAX_SETS, max(1, -(-2 * L2_BYTES // int(bytes_apply + 1)))))
+    x = [torch.randn(d, device=dev) for _ in range(n_x)]
+    bits = [torch.zeros(M, ldw, dtype=torch.int32, device=dev) for _ in range(n_sets)]
+    vote = [torch.zeros(W, dtype=torch.int32, device=dev) for _ in range(max(n_sets, n_x))]
+    for s in range(n_sets):                                  # realistic bit rows for the vote
+        B.sign_pack(g[s % n_sets_big], M, d, ld, bits[s], ldw)
+    rows = []
+
+    def rec(name, ms, nbytes, cold):
+        gbs = nbytes / (ms * 1e-3) / 1e9
+        rows.append((d, M, name, ms * 1e3, gbs, gbs / peak_gbs(), int(cold)))
+
+    ms = time_launches(lambda s: B.signum_momentum_pack(g[s % n_sets_big], m[s % n_sets_big], M, d, ld, beta,
+                                                        bits[s % n_sets], ldw), n_sets_big, reps)
+    rec("momentum_pack", ms, bytes_worker, n_sets_big * bytes_worker >= 2 * L2_BYTES)
+    ms = time_launches(lambda s: B.majority_vote(bits[s], M, d, ldw, vote[s]), n_sets, reps)
+    rec("majority_vote", ms, bytes_vote, n_sets * bytes_vote >= 2 * L2_BYTES)
+    ms = time_launches(lambda s: B.sign_apply(x[s], vote[s], d, delta), n_x, reps)
+    rec("sign_apply", ms, bytes_apply, n_x * bytes_apply >= 2 * L2_BYTES)
+    ms = time_launches(lambda s: B.signsgd_step(x[s % n_x], g[s % n_sets_big], m[s % n_sets_big], M, d, ld, beta,
+                                                delta, bits[s % n_sets], ldw, vote[s % n_sets]),
+                       n_sets_big, reps)
+    rec("signsgd_step", ms, bytes_worker + bytes_apply, n_sets_big * bytes_worker >= 2 * L2_BYTES)
+    return rows
+
+
+def main(argv=None):
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--min-log2", type=int, default=10)
+    ap.add_argument("--max-log2", type=int, default=28)
+    ap.add_argument("--workers", default="1,3,7,15,31")
+    ap.add_argument("--reps", type=int, default=20)
+    ap.add_argument("--out", default=None)
+    args = ap.parse_args(argv)
+    if not torch.cuda.is_available():
+        raise SystemExit("the sweep needs a CUDA device")
+    dev = torch.device("cuda", 0)
+    B.lib()
+    out = open(args.out, "w") if args.out else None
+    header = "d\tM\tkernel\tus_per_launch\talgorithmic_GBps\tfrac_of_measured_peak\tcold"
+    print(header)
+    if out:
+        out.write(header + "\n")
+    for M in [int(t) for t in args.workers.split(",")]:
+        for k in range(args.min_log2, args.max_log2 + 1):
+            reps = args.reps if k < 24 else max(2, args.reps // 8)
+            for r in run_point(1 << k, M, reps, dev):
+                line = "%d\t%d\t%s\t%.2f\t%.1f\t%.3f\t%d" % r
+                print(line, flush=True)
+                if out:
+                    out.write(line + "\n")
+            torch.cuda.empty_cache()
+    if out:
+        out.close()
+
+
+if __name__ == "__main__":
+    sys.exit(main())
