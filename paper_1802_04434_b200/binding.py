@@ -18,6 +18,7 @@ import torch
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libsignsgd_b200.so")
 MAX_WORKERS = 1024
+FUSED_MAX_WORKERS = 8      # ssgd_signsgd_step runs as one fused kernel up to this many workers
 
 _lib = None
 

@@ -378,9 +378,100 @@ apply_kernel(float* __restrict__ x, const uint32_t* __restrict__ vote, unsigned 
 // and folds it into a private bit-sliced counter.  After the last row the top
 // plane of that counter is the voted word; it is stored and handed back to the
 // eight lanes of its group by shuffles for the update of x.
+//
+// Measured on B200: with few workers (M <= 8) this beats the three separate
+// kernels (one launch, no second pass over the words); with many workers the
+// 2M + 1 concurrent row streams cost 1-5 % of DRAM efficiency against the worker
+// kernel's two, so the step entry point then uses the three kernels.
+
+constexpr int kFusedMaxWorkers = 8;   // rows walked by one CTA at most
+constexpr int kFusedMaxPlanes = 4;    // planes needed for M <= 8
 
 template <bool MOMENTUM, int UNROLL, int NP>
-__global__ void __launch_bounds__(kThreads)
+__device__ __forceinline__ void fused_row(const float* __restrict__ gr, float* __restrict__ mr,
+                                          uint32_t* __restrict__ brow, float beta, float omb,
+                                          unsigned lane, unsigned sub, unsigned long long my_word,
+                                          Counter1<NP>& cnt) {
+  float4 gv[UNROLL], mv[UNROLL];
+#pragma unroll
+  for (int u = 0; u < UNROLL; ++u) gv[u] = ld128(gr + u * 128);
+  if (MOMENTUM) {
+#pragma unroll
+    for (int u = 0; u < UNROLL; ++u) mv[u] = ld128(mr + u * 128);
+  }
+  unsigned mine = 0;
+#pragma unroll
+  for (int u = 0; u < UNROLL; ++u) {
+    float4 v = gv[u];
+    if (MOMENTUM) {
+      v = momentum_update4(beta, omb, mv[u], v);
+      st128(mr + u * 128, v);
+    }
+    const unsigned word = assemble_word(sign_nibble(v), lane);
+    if (sub == (unsigned)u) mine = word;
+  }
+  if (sub < (unsigned)UNROLL) brow[my_word] = mine;
+  cnt.template add<0>(mine);
+}
+
+// The span that crosses the end of the vector: the same walk with element-wise
+// guards.  Bits at positions >= d stay 0 in every row, so they count 0 votes and
+// the voted word has them 0 as well (the threshold is at least 1).  Kept out of
+// line so that the interior path's register allocation is not affected.
+template <bool MOMENTUM, int UNROLL, int NP>
+__device__ __noinline__ void fused_ragged_span(const float* __restrict__ g, float* __restrict__ m,
+                                               float* __restrict__ x, uint32_t* __restrict__ bits,
+                                               uint32_t* __restrict__ vote, unsigned M,
+                                               unsigned long long d, unsigned long long ld,
+                                               unsigned long long ldw, float beta, float omb, float delta,
+                                               unsigned start_value, unsigned long long e0) {
+  const unsigned lane = threadIdx.x & 31u;
+  const unsigned sub = lane & 7u;
+  const float minus = -delta;
+  const unsigned long long my_word = (e0 >> 5) + own_word_index<UNROLL>(lane);
+  const bool have_word = sub < (unsigned)UNROLL && my_word * 32 < d;   // its first element is below d
+  Counter1<NP> cnt;
+  cnt.init(start_value);
+  for (unsigned row = 0; row < M; ++row) {
+    const float* gr = g + (unsigned long long)row * ld;
+    float* mr = MOMENTUM ? m + (unsigned long long)row * ld : nullptr;
+    unsigned mine = 0;
+#pragma unroll 1
+    for (int u = 0; u < UNROLL; ++u) {
+      const unsigned long long e = e0 + u * 128 + lane * 4;
+      unsigned nib = 0;
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        if (e + k < d) {
+          float v = gr[e + k];
+          if (MOMENTUM) {
+            v = momentum_update(beta, omb, mr[e + k], v);
+            mr[e + k] = v;
+          }
+          nib |= sign_bit(v) << k;
+        }
+      }
+      const unsigned word = assemble_word(nib, lane);
+      if (sub == (unsigned)u) mine = word;
+    }
+    if (have_word) bits[(unsigned long long)row * ldw + my_word] = mine;
+    cnt.template add<0>(mine);
+  }
+  const unsigned voted = cnt.top();
+  if (have_word) vote[my_word] = voted;
+#pragma unroll 1
+  for (int u = 0; u < UNROLL; ++u) {
+    const unsigned vw = __shfl_sync(0xFFFFFFFFu, voted, (lane & 24u) + u);
+    const unsigned long long e = e0 + u * 128 + lane * 4;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      if (e + k < d) x[e + k] = __fadd_rn(x[e + k], ((vw >> (4u * sub + k)) & 1u) ? minus : delta);
+    }
+  }
+}
+
+template <bool MOMENTUM, int UNROLL, int NP>
+__global__ void __launch_bounds__(kThreads, 5)
 fused_step_kernel(const float* __restrict__ g, float* __restrict__ m, float* __restrict__ x,
                   uint32_t* __restrict__ bits, uint32_t* __restrict__ vote, unsigned M,
                   unsigned long long d, unsigned long long ld, unsigned long long ldw,
@@ -390,92 +481,32 @@ fused_step_kernel(const float* __restrict__ g, float* __restrict__ m, float* __r
   const unsigned lane = threadIdx.x & 31u;
   const unsigned warp = threadIdx.x >> 5;
   const unsigned sub = lane & 7u;
-  const float minus = -delta;
   const unsigned long long e0 = (unsigned long long)blockIdx.x * TILE + (unsigned long long)warp * SPAN;
   if (e0 >= d) return;   // uniform over the warp; nothing below synchronises across warps
-
+  if (e0 + SPAN > d) {
+    fused_ragged_span<MOMENTUM, UNROLL, NP>(g, m, x, bits, vote, M, d, ld, ldw, beta, omb, delta,
+                                            start_value, e0);
+    return;
+  }
   Counter1<NP> cnt;
   cnt.init(start_value);
-  const unsigned long long w0 = e0 >> 5;                      // first word of the span
-  const unsigned long long my_word = w0 + own_word_index<UNROLL>(lane);
-
-  if (e0 + SPAN <= d) {
-    const unsigned long long off = e0 + lane * 4;
-    for (unsigned row = 0; row < M; ++row) {
-      const float* gr = g + (unsigned long long)row * ld + off;
-      float* mr = MOMENTUM ? m + (unsigned long long)row * ld + off : nullptr;
-      float4 gv[UNROLL], mv[UNROLL];
+  const unsigned long long my_word = (e0 >> 5) + own_word_index<UNROLL>(lane);
+  const unsigned long long off = e0 + lane * 4;
+  for (unsigned row = 0; row < M; ++row) {
+    fused_row<MOMENTUM, UNROLL, NP>(g + (unsigned long long)row * ld + off,
+                                    MOMENTUM ? m + (unsigned long long)row * ld + off : nullptr,
+                                    bits + (unsigned long long)row * ldw, beta, omb, lane, sub, my_word, cnt);
+  }
+  const unsigned voted = cnt.top();
+  if (sub < (unsigned)UNROLL) vote[my_word] = voted;
+  const float minus = -delta;
+  float4 xv[UNROLL];
 #pragma unroll
-      for (int u = 0; u < UNROLL; ++u) gv[u] = ld128(gr + u * 128);
-      if (MOMENTUM) {
+  for (int u = 0; u < UNROLL; ++u) xv[u] = ld128(x + off + u * 128);
 #pragma unroll
-        for (int u = 0; u < UNROLL; ++u) mv[u] = ld128(mr + u * 128);
-      }
-      unsigned mine = 0;
-#pragma unroll
-      for (int u = 0; u < UNROLL; ++u) {
-        float4 v = gv[u];
-        if (MOMENTUM) {
-          v = momentum_update4(beta, omb, mv[u], v);
-          st128(mr + u * 128, v);
-        }
-        const unsigned word = assemble_word(sign_nibble(v), lane);
-        if (sub == (unsigned)u) mine = word;
-      }
-      if (sub < (unsigned)UNROLL) bits[(unsigned long long)row * ldw + my_word] = mine;
-      cnt.template add<0>(mine);
-    }
-    const unsigned voted = cnt.top();
-    if (sub < (unsigned)UNROLL) vote[my_word] = voted;
-    float4 xv[UNROLL];
-#pragma unroll
-    for (int u = 0; u < UNROLL; ++u) xv[u] = ld128(x + off + u * 128);
-#pragma unroll
-    for (int u = 0; u < UNROLL; ++u) {
-      const unsigned vw = __shfl_sync(0xFFFFFFFFu, voted, (lane & 24u) + u);  // owner of step u in my group
-      st128(x + off + u * 128, apply4(xv[u], vw >> (4u * sub), delta, minus));
-    }
-  } else {
-    // ragged end of the vector: the same walk with element-wise guards.  Bits at
-    // positions >= d stay 0 in every row, so they count 0 votes and the voted
-    // word has them 0 as well (the threshold is at least 1).
-    for (unsigned row = 0; row < M; ++row) {
-      const float* gr = g + (unsigned long long)row * ld;
-      float* mr = MOMENTUM ? m + (unsigned long long)row * ld : nullptr;
-      unsigned mine = 0;
-#pragma unroll 1
-      for (int u = 0; u < UNROLL; ++u) {
-        const unsigned long long e = e0 + u * 128 + lane * 4;
-        unsigned nib = 0;
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-          if (e + k < d) {
-            float v = gr[e + k];
-            if (MOMENTUM) {
-              v = momentum_update(beta, omb, mr[e + k], v);
-              mr[e + k] = v;
-            }
-            nib |= sign_bit(v) << k;
-          }
-        }
-        const unsigned word = assemble_word(nib, lane);
-        if (sub == (unsigned)u) mine = word;
-      }
-      // my word exists iff its first element is below d
-      if (sub < (unsigned)UNROLL && my_word * 32 < d) bits[(unsigned long long)row * ldw + my_word] = mine;
-      cnt.template add<0>(mine);
-    }
-    const unsigned voted = cnt.top();
-    if (sub < (unsigned)UNROLL && my_word * 32 < d) vote[my_word] = voted;
-#pragma unroll 1
-    for (int u = 0; u < UNROLL; ++u) {
-      const unsigned vw = __shfl_sync(0xFFFFFFFFu, voted, (lane & 24u) + u);
-      const unsigned long long e = e0 + u * 128 + lane * 4;
-#pragma unroll
-      for (int k = 0; k < 4; ++k) {
-        if (e + k < d) x[e + k] = __fadd_rn(x[e + k], ((vw >> (4u * sub + k)) & 1u) ? minus : delta);
-      }
-    }
+  for (int u = 0; u < UNROLL; ++u) {
+    const unsigned vw = __shfl_sync(0xFFFFFFFFu, voted, (lane & 24u) + u);  // owner of step u in my group
+    st128(x + off + u * 128, apply4(xv[u], vw >> (4u * sub), delta, minus));
   }
 }
 
@@ -645,33 +676,23 @@ bool launch_fused_mu(const StepArgs& a, cudaStream_t s) {
     case 2: launch_fused_mun<MOMENTUM, UNROLL, 2>(a, s); return true;
     case 3: launch_fused_mun<MOMENTUM, UNROLL, 3>(a, s); return true;
     case 4: launch_fused_mun<MOMENTUM, UNROLL, 4>(a, s); return true;
-    case 5: launch_fused_mun<MOMENTUM, UNROLL, 5>(a, s); return true;
-    case 6: launch_fused_mun<MOMENTUM, UNROLL, 6>(a, s); return true;
-    case 7: launch_fused_mun<MOMENTUM, UNROLL, 7>(a, s); return true;
-    case 8: launch_fused_mun<MOMENTUM, UNROLL, 8>(a, s); return true;
-    case 9: launch_fused_mun<MOMENTUM, UNROLL, 9>(a, s); return true;
-    case 10: launch_fused_mun<MOMENTUM, UNROLL, 10>(a, s); return true;
-    case 11: launch_fused_mun<MOMENTUM, UNROLL, 11>(a, s); return true;
   }
   return false;
 }
 
-// The fused kernel's grid is one CTA per tile of columns; vectors too long for
-// one grid (beyond 2^31 tiles) take the three-kernel path instead.
+// Whether the step runs as the fused kernel: few workers, and a vector that fits
+// one grid of tiles.  Everything else takes the three kernels.
 template <bool MOMENTUM>
 ssgd_status launch_fused(const StepArgs& a, cudaStream_t s, bool* launched) {
+  static_assert(kFusedMaxWorkers / 2 < (1 << (kFusedMaxPlanes - 1)), "planes cover the fused worker limit");
+  *launched = false;
+  if (a.M > (size_t)kFusedMaxWorkers) return SSGD_OK;
   DeviceInfo di;
   if (!device_info(&di)) return SSGD_ERR_CUDA;
-  const int unroll = pick_unroll(a.d, 1, di.sms);
+  const int unroll = pick_unroll(a.d, 1, di.sms) >= 2 ? 2 : 1;
   const unsigned long long tile = (unsigned long long)kThreads * 4 * unroll;
-  *launched = false;
   if ((a.d + tile - 1) / tile > kMaxGrid) return SSGD_OK;
-  bool ok;
-  switch (unroll) {
-    case 4: ok = launch_fused_mu<MOMENTUM, 4>(a, s); break;
-    case 2: ok = launch_fused_mu<MOMENTUM, 2>(a, s); break;
-    default: ok = launch_fused_mu<MOMENTUM, 1>(a, s); break;
-  }
+  const bool ok = unroll == 2 ? launch_fused_mu<MOMENTUM, 2>(a, s) : launch_fused_mu<MOMENTUM, 1>(a, s);
   if (!ok) return SSGD_ERR_SIZE;
   *launched = true;
   return launch_status();
@@ -781,7 +802,7 @@ ssgd_status ssgd_signsgd_step(float* x, const float* g, float* m, size_t M, size
   bool launched = false;
   st = m ? launch_fused<true>(a, s, &launched) : launch_fused<false>(a, s, &launched);
   if (st != SSGD_OK || launched) return st;
-  // vectors beyond one grid of tiles: the same step as three launches
+  // many workers, or a vector beyond one grid of tiles: the same step as three launches
   st = m ? launch_worker<true>(g, m, M, d, ld, beta, bits_ws, ldw, s)
          : launch_worker<false>(g, nullptr, M, d, ld, 0.0f, bits_ws, ldw, s);
   if (st != SSGD_OK) return st;
