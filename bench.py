@@ -33,9 +33,9 @@ FALLBACK_HBM_GBS = 6650.0
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the dominant kernel,
 # from the ncu capture summarised in profiles/; valid only while the kernel source is unchanged.
 NCU_TRAFFIC = {
-    "source_sha256": "0582867d44a66a4250c708e3ce49e3acf2d6ec1cecc4f52835e211f6347fa7ac",
+    "source_sha256": "1d19a1aa35982188ce470bf7a08d9b771fa5978bc3f1345996562d5dd8a19bb2",
     "workload": "resnet50_d25557056_M7",
-    "bytes_per_launch": 1.431786e9 + 683.192832e6,
+    "bytes_per_launch": 1.533631e9 + 792.701952e6,
 }
 
 
@@ -212,23 +212,19 @@ def workload_config(cfg, n_gpus):
 
 def run_ours(args):
     import torch
-    import torch.distributed as dist
     from paper_1802_04434_b200 import binding as B
+    from paper_1802_04434_b200 import multi
 
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank, local_rank, world = multi.env_ranks()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
-    if world > 1:
-        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
-        dist.init_process_group("nccl", device_id=dev)
+    multi.init(dev)
     B.lib()  # fail here, loudly, if the CUDA library is missing
 
     cfg = get_workload(args.workload)
-    cfg.seed = rank            # every rank owns an independent shard of a larger vector
+    cfg.seed = multi.shard_seed(rank)   # every rank owns an independent shard of a larger vector
     M, d, ld, ldw, W = cfg.M, cfg.d, cfg.ld, cfg.ldw, cfg.words
     momentum = cfg.momentum_buffer
     shared = cfg.shared(dev)
@@ -261,9 +257,7 @@ def run_ours(args):
         B.sign_apply(x, vote, d, cfg.delta, stream)
 
     def barrier():
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
+        multi.barrier(dev)
 
     K, Wm = args.steps, args.warmup
     events = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
@@ -294,11 +288,8 @@ def run_ours(args):
         sampler.stop()
     worker_ms = sum(a.elapsed_time(b) for a, b in events) / K
 
-    if world > 1:
-        t = torch.tensor([elapsed_ms, worker_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        elapsed_ms, worker_ms = float(t[0]), float(t[1])
-    value = world * d * K / (elapsed_ms * 1e-3)
+    elapsed_ms, worker_ms = multi.max_over_ranks([elapsed_ms, worker_ms], dev)
+    value = multi.whole_job_rate(d, K, elapsed_ms, world)
     ms_per_step = elapsed_ms / K
 
     # end to end through the host-buffer entry point: gradients start in pinned host memory,
@@ -317,11 +308,8 @@ def run_ours(args):
     e1.record(stream)
     barrier()
     e2e_ms = e0.elapsed_time(e1)
-    if world > 1:
-        t = torch.tensor([e2e_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t[0])
-    e2e_value = world * d * Ke / (e2e_ms * 1e-3)
+    (e2e_ms,) = multi.max_over_ranks([e2e_ms], dev)
+    e2e_value = multi.whole_job_rate(d, Ke, e2e_ms, world)
 
     if rank == 0:
         peak, peak_kind = measured_peak()
@@ -354,8 +342,7 @@ def run_ours(args):
             line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle",
                                     "sample": "first %d of %d elements, M=%d, 3 steps, single thread" % (n, d, M)}
         print(json.dumps(line), flush=True)
-    if world > 1:
-        dist.destroy_process_group()
+    multi.finish()
 
 
 def main():

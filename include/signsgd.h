@@ -115,6 +115,50 @@ ssgd_status ssgd_signsgd_step(float* x, const float* g, float* m, size_t M,
                               uint32_t* bits_ws, size_t ldw, uint32_t* vote_ws,
                               void* stream);
 
+/* Theorem 3 (Signum): the warm-up length C(beta), the least positive integer C
+ * with (C/2) beta^C <= 1 / ((1 - beta^2)(C + 1)) and beta^(C+1) <= 1/2; the
+ * paper notes C(0.9) = 54.  Pure host arithmetic, no GPU work.  Returns 0 when
+ * beta is outside [0,1) or NaN.  The scan takes about 5/(1-beta) iterations. */
+size_t ssgd_warmup_steps(float beta);
+
+/* Theorem 3's warm-up iteration on the worker side: "accumulate the momentum as
+ * normal, but use the sign of the stochastic gradient to make updates".  Same as
+ * ssgd_signum_momentum_pack (m updated in place, identical values) except that
+ * bit i of row w = !(g[w][i] < 0), the words of ssgd_sign_pack.               */
+ssgd_status ssgd_signum_warmup_pack(const float* g, float* m, size_t M, size_t d,
+                                    size_t ld, float beta, uint32_t* bits,
+                                    size_t ldw, void* stream);
+
+/* One whole warm-up step: ssgd_signum_warmup_pack for all M workers, majority
+ * vote, apply.  Arguments as ssgd_signsgd_step; m is required.  A training loop
+ * calls this for iterations k < ssgd_warmup_steps(beta) and ssgd_signsgd_step
+ * afterwards.                                                                  */
+ssgd_status ssgd_signsgd_warmup_step(float* x, const float* g, float* m, size_t M,
+                                     size_t d, size_t ld, float beta, float delta,
+                                     uint32_t* bits_ws, size_t ldw,
+                                     uint32_t* vote_ws, void* stream);
+
+/* The "(good)" scheme of Section 4, x <- x - delta * sum_m sign(g_m): the server
+ * sends back the vote COUNT instead of its sign, so the way down is no longer
+ * 1-bit.  Here the count travels bit-sliced:
+ *   counts uint32 [ssgd_count_planes(M)][ldc]: bit k of word j of plane p is bit
+ *   p of P_(32j+k), the number of workers whose bit for parameter 32j+k is set
+ *   (0 <= P <= M); ldc a multiple of 4, ldc >= W; bits at positions >= d are 0.
+ * ssgd_count_planes(M) = bit length of M (planes needed for 0..M); 0 if M is
+ * out of range.                                                               */
+size_t ssgd_count_planes(size_t M);
+
+/* Server side of the "(good)" scheme: count the +1 votes per parameter.
+ *   bits in [M][ldw]; counts out [ssgd_count_planes(M)][ldc].                  */
+ssgd_status ssgd_vote_counts(const uint32_t* bits, size_t M, size_t d, size_t ldw,
+                             uint32_t* counts, size_t ldc, void* stream);
+
+/* Worker side of the "(good)" scheme: with S = 2 P - M the sum of the M signs,
+ *   x[i] <- fma(-delta, (float)S_i, x[i])       (one fp32 rounding), in place.
+ * The sign of S is the majority vote (S = 0 being the tie).                    */
+ssgd_status ssgd_sum_apply(float* x, const uint32_t* counts, size_t M, size_t d,
+                           size_t ldc, float delta, void* stream);
+
 /* ssgd_signsgd_step for a caller whose gradients live in HOST memory
  * (Algorithm 3's "independent gradient estimate" arriving from outside the
  * device): copies g_host to the device staging buffer, runs the step, and

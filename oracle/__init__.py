@@ -47,6 +47,10 @@ def _load():
     sz, f32, vp = ctypes.c_size_t, ctypes.c_float, ctypes.c_void_p
     L.ssgd_words_ref.restype = sz
     L.ssgd_words_ref.argtypes = [sz]
+    L.ssgd_count_planes_ref.restype = sz
+    L.ssgd_count_planes_ref.argtypes = [sz]
+    L.ssgd_warmup_steps_ref.restype = sz
+    L.ssgd_warmup_steps_ref.argtypes = [f32]
     for name, args in {
         "ssgd_sign_unpacked_ref": [vp, sz, vp],
         "ssgd_pack_bits_ref": [vp, sz, vp],
@@ -54,7 +58,11 @@ def _load():
         "ssgd_sign_pack_ref": [vp, sz, sz, sz, vp, sz],
         "ssgd_momentum_ref": [vp, vp, sz, f32],
         "ssgd_signum_momentum_pack_ref": [vp, vp, sz, sz, sz, f32, vp, sz],
+        "ssgd_signum_warmup_pack_ref": [vp, vp, sz, sz, sz, f32, vp, sz],
+        "ssgd_signsgd_warmup_step_ref": [vp, vp, vp, sz, sz, sz, f32, f32, vp, sz, vp],
         "ssgd_vote_counts_ref": [vp, sz, sz, sz, vp],
+        "ssgd_vote_count_planes_ref": [vp, sz, sz, sz, vp, sz],
+        "ssgd_sum_apply_ref": [vp, vp, sz, sz, sz, f32],
         "ssgd_majority_vote_ref": [vp, sz, sz, sz, vp],
         "ssgd_sign_apply_ref": [vp, vp, sz, f32],
         "ssgd_signsgd_step_ref": [vp, vp, vp, sz, sz, sz, f32, f32, vp, sz, vp],
@@ -179,3 +187,58 @@ def signsgd_step(x: np.ndarray, g: np.ndarray, m: np.ndarray | None, M: int, d: 
         _chk(x, np.float32, d, "x", True), _chk(g, np.float32, M * ld, "g"), mp,
         M, d, ld, beta, delta, bits.ctypes.data, ldw, vote.ctypes.data)
     return bits, vote
+
+
+def warmup_steps(beta: float) -> int:
+    """C(beta) of Theorem 3 (the paper notes C(0.9) = 54)."""
+    return int(_load().ssgd_warmup_steps_ref(beta))
+
+
+def signum_warmup_pack(g: np.ndarray, m: np.ndarray, M: int, d: int, beta: float,
+                       ld: int | None = None, ldw: int | None = None) -> np.ndarray:
+    """Theorem 3 warm-up on the worker: m updated as in Algorithm 2, returns packed sign(g)."""
+    ld, ldw = _rows(M, d, ld, ldw)
+    bits = np.zeros(M * ldw, dtype=np.uint32)
+    _load().ssgd_signum_warmup_pack_ref(
+        _chk(g, np.float32, M * ld, "g"), _chk(m, np.float32, M * ld, "m", True),
+        M, d, ld, beta, bits.ctypes.data, ldw)
+    return bits
+
+
+def signsgd_warmup_step(x: np.ndarray, g: np.ndarray, m: np.ndarray, M: int, d: int,
+                        beta: float, delta: float, ld: int | None = None,
+                        ldw: int | None = None):
+    """One whole warm-up step; returns (bits, vote)."""
+    ld, ldw = _rows(M, d, ld, ldw)
+    bits = np.zeros(M * ldw, dtype=np.uint32)
+    vote = np.empty(words(d), dtype=np.uint32)
+    _load().ssgd_signsgd_warmup_step_ref(
+        _chk(x, np.float32, d, "x", True), _chk(g, np.float32, M * ld, "g"),
+        _chk(m, np.float32, M * ld, "m", True), M, d, ld, beta, delta,
+        bits.ctypes.data, ldw, vote.ctypes.data)
+    return bits, vote
+
+
+def count_planes(M: int) -> int:
+    """Bit planes needed for a vote count in 0..M."""
+    return int(_load().ssgd_count_planes_ref(M))
+
+
+def vote_count_planes(bits: np.ndarray, M: int, d: int, ldw: int | None = None,
+                      ldc: int | None = None) -> np.ndarray:
+    """Server side of the "(good)" scheme (Sec. 4): bit-sliced counts of +1 votes, [planes][ldc]."""
+    _, ldw = _rows(M, d, None, ldw)
+    ldc = words(d) if ldc is None else ldc
+    out = np.zeros(count_planes(M) * ldc, dtype=np.uint32)
+    _load().ssgd_vote_count_planes_ref(_chk(bits, np.uint32, M * ldw, "bits"), M, d, ldw,
+                                       out.ctypes.data, ldc)
+    return out
+
+
+def sum_apply(x: np.ndarray, counts: np.ndarray, M: int, d: int, delta: float,
+              ldc: int | None = None) -> None:
+    """Worker side of the "(good)" scheme: x <- x - delta * sum_m sign(.), in place."""
+    ldc = words(d) if ldc is None else ldc
+    _load().ssgd_sum_apply_ref(_chk(x, np.float32, d, "x", True),
+                               _chk(counts, np.uint32, count_planes(M) * ldc, "counts"),
+                               M, d, ldc, delta)

@@ -93,6 +93,32 @@ void ssgd_signum_momentum_pack_ref(const float* g, float* m, size_t M, size_t d,
   }
 }
 
+// Theorem 3's warm-up length: C(beta) = min C in Z+ such that
+//   (C/2) beta^C <= 1/(1 - beta^2) * 1/(C + 1)   and   beta^(C+1) <= 1/2.
+// Each candidate is tested directly from this definition, in extended precision.
+size_t ssgd_warmup_steps_ref(float beta) {
+  if (!(beta >= 0.0f && beta < 1.0f)) return 0;
+  const long double b = (long double)beta;
+  for (size_t C = 1;; ++C) {
+    const long double lhs = ((long double)C / 2.0L) * std::pow(b, (long double)C);
+    const long double rhs = 1.0L / (1.0L - b * b) * 1.0L / ((long double)C + 1.0L);
+    if (lhs <= rhs && std::pow(b, (long double)C + 1.0L) <= 0.5L) return C;
+  }
+}
+
+// Theorem 3, warm-up iterations: the momentum is accumulated as in Algorithm 2,
+// but the sign that is sent is that of the stochastic gradient.
+void ssgd_signum_warmup_pack_ref(const float* g, float* m, size_t M, size_t d,
+                                 size_t ld, float beta, uint32_t* bits,
+                                 size_t ldw) {
+  std::vector<uint8_t> s(d);
+  for (size_t w = 0; w < M; ++w) {
+    ssgd_momentum_ref(g + w * ld, m + w * ld, d, beta);
+    ssgd_sign_unpacked_ref(g + w * ld, d, s.data());
+    ssgd_pack_bits_ref(s.data(), d, bits + w * ldw);
+  }
+}
+
 // Algorithm 3 server side on unpacked signs: count the +1 votes per element.
 void ssgd_vote_counts_ref(const uint32_t* bits, size_t M, size_t d, size_t ldw,
                           int32_t* P) {
@@ -139,6 +165,53 @@ void ssgd_signsgd_step_ref(float* x, const float* g, float* m, size_t M,
   } else {
     ssgd_signum_momentum_pack_ref(g, m, M, d, ld, beta, bits, ldw);
   }
+  ssgd_majority_vote_ref(bits, M, d, ldw, vote);
+  ssgd_sign_apply_ref(x, vote, d, delta);
+}
+
+// ---- the "(good)" scheme of Section 4: x <- x - delta * sum_m sign(g_m) --------
+// The server's answer is the count P of +1 votes per element (sum of signs =
+// 2P - M), sent bit-sliced: plane p holds bit p of every count, packed like a
+// sign vector.
+
+size_t ssgd_count_planes_ref(size_t M) {
+  size_t n = 0;
+  while ((M >> n) != 0) ++n;   // bits needed for the values 0..M
+  return n;
+}
+
+void ssgd_vote_count_planes_ref(const uint32_t* bits, size_t M, size_t d,
+                                size_t ldw, uint32_t* counts, size_t ldc) {
+  std::vector<int32_t> P(d);
+  std::vector<uint8_t> s(d);
+  ssgd_vote_counts_ref(bits, M, d, ldw, P.data());
+  const size_t planes = ssgd_count_planes_ref(M);
+  for (size_t p = 0; p < planes; ++p) {
+    for (size_t i = 0; i < d; ++i) s[i] = uint8_t((P[i] >> p) & 1);
+    ssgd_pack_bits_ref(s.data(), d, counts + p * ldc);
+  }
+}
+
+void ssgd_sum_apply_ref(float* x, const uint32_t* counts, size_t M, size_t d,
+                        size_t ldc, float delta) {
+  const size_t planes = ssgd_count_planes_ref(M);
+  std::vector<uint8_t> s(d);
+  std::vector<int32_t> P(d, 0);
+  for (size_t p = 0; p < planes; ++p) {
+    ssgd_unpack_bits_ref(counts + p * ldc, d, s.data());
+    for (size_t i = 0; i < d; ++i) P[i] += int32_t(s[i]) << p;
+  }
+  for (size_t i = 0; i < d; ++i) {
+    const float sum_of_signs = float(2 * P[i] - int32_t(M));
+    x[i] = std::fmaf(-delta, sum_of_signs, x[i]);   // x - delta * sum, rounded once
+  }
+}
+
+// One whole warm-up step: Theorem 3's warm-up on every worker, then Algorithm 3.
+void ssgd_signsgd_warmup_step_ref(float* x, const float* g, float* m, size_t M,
+                                  size_t d, size_t ld, float beta, float delta,
+                                  uint32_t* bits, size_t ldw, uint32_t* vote) {
+  ssgd_signum_warmup_pack_ref(g, m, M, d, ld, beta, bits, ldw);
   ssgd_majority_vote_ref(bits, M, d, ldw, vote);
   ssgd_sign_apply_ref(x, vote, d, delta);
 }

@@ -42,6 +42,10 @@ def lib() -> ctypes.CDLL:
     sz, f32, vp, ci = ctypes.c_size_t, ctypes.c_float, ctypes.c_void_p, ctypes.c_int
     L.ssgd_words.restype = sz
     L.ssgd_words.argtypes = [sz]
+    L.ssgd_count_planes.restype = sz
+    L.ssgd_count_planes.argtypes = [sz]
+    L.ssgd_warmup_steps.restype = sz
+    L.ssgd_warmup_steps.argtypes = [f32]
     L.ssgd_status_str.restype = ctypes.c_char_p
     L.ssgd_status_str.argtypes = [ci]
     sigs = {
@@ -50,6 +54,10 @@ def lib() -> ctypes.CDLL:
         "ssgd_majority_vote": [vp, sz, sz, sz, vp, vp],
         "ssgd_sign_apply": [vp, vp, sz, f32, vp],
         "ssgd_signsgd_step": [vp, vp, vp, sz, sz, sz, f32, f32, vp, sz, vp, vp],
+        "ssgd_signum_warmup_pack": [vp, vp, sz, sz, sz, f32, vp, sz, vp],
+        "ssgd_signsgd_warmup_step": [vp, vp, vp, sz, sz, sz, f32, f32, vp, sz, vp, vp],
+        "ssgd_vote_counts": [vp, sz, sz, sz, vp, sz, vp],
+        "ssgd_sum_apply": [vp, vp, sz, sz, sz, f32, vp],
         "ssgd_signsgd_step_host": [vp, vp, vp, sz, sz, sz, f32, f32, vp, vp, sz, vp, vp, vp],
         "ssgd_signsgd_step_noalloc": [vp, vp, vp, sz, sz, sz, f32, f32, vp],
     }
@@ -149,6 +157,54 @@ def signsgd_step(x: torch.Tensor, g: torch.Tensor, m: Optional[torch.Tensor], M:
         _ptr(x, torch.float32, "x"), _ptr(g, torch.float32, "g"), _ptr(m, torch.float32, "m"),
         M, d, ld, beta, delta, _ptr(bits_ws, WORD_DTYPE, "bits_ws"), ldw,
         _ptr(vote_ws, WORD_DTYPE, "vote_ws"), _stream(stream)), "ssgd_signsgd_step")
+
+
+def warmup_steps(beta: float) -> int:
+    """C(beta) of Theorem 3: how many warm-up iterations Signum's analysis asks for (54 at 0.9)."""
+    return int(lib().ssgd_warmup_steps(beta))
+
+
+def signum_warmup_pack(g: torch.Tensor, m: torch.Tensor, M: int, d: int, ld: int, beta: float,
+                       bits: torch.Tensor, ldw: int, stream=None) -> None:
+    """Warm-up worker step of Theorem 3: m updated as in Algorithm 2, bits <- sign(g)."""
+    _need(g, M * ld, "g"); _need(m, M * ld, "m"); _need(bits, M * ldw, "bits")
+    _check(lib().ssgd_signum_warmup_pack(
+        _ptr(g, torch.float32, "g"), _ptr(m, torch.float32, "m"), M, d, ld, beta,
+        _ptr(bits, WORD_DTYPE, "bits"), ldw, _stream(stream)), "ssgd_signum_warmup_pack")
+
+
+def signsgd_warmup_step(x: torch.Tensor, g: torch.Tensor, m: torch.Tensor, M: int, d: int, ld: int,
+                        beta: float, delta: float, bits_ws: torch.Tensor, ldw: int,
+                        vote_ws: torch.Tensor, stream=None) -> None:
+    """One whole warm-up step (momentum accumulates, the vote is over sign(g))."""
+    _need(x, d, "x"); _need(g, M * ld, "g"); _need(m, M * ld, "m")
+    _need(bits_ws, M * ldw, "bits_ws"); _need(vote_ws, -(-d // 32), "vote_ws")
+    _check(lib().ssgd_signsgd_warmup_step(
+        _ptr(x, torch.float32, "x"), _ptr(g, torch.float32, "g"), _ptr(m, torch.float32, "m"),
+        M, d, ld, beta, delta, _ptr(bits_ws, WORD_DTYPE, "bits_ws"), ldw,
+        _ptr(vote_ws, WORD_DTYPE, "vote_ws"), _stream(stream)), "ssgd_signsgd_warmup_step")
+
+
+def count_planes(M: int) -> int:
+    """Bit planes that hold a vote count 0..M (the bit length of M)."""
+    return int(lib().ssgd_count_planes(M))
+
+
+def vote_counts(bits: torch.Tensor, M: int, d: int, ldw: int, counts: torch.Tensor, ldc: int,
+                stream=None) -> None:
+    """Server side of the "(good)" scheme of Sec. 4: bit-sliced number of +1 votes per parameter."""
+    _need(bits, M * ldw, "bits"); _need(counts, count_planes(M) * ldc, "counts")
+    _check(lib().ssgd_vote_counts(_ptr(bits, WORD_DTYPE, "bits"), M, d, ldw,
+                                  _ptr(counts, WORD_DTYPE, "counts"), ldc, _stream(stream)),
+           "ssgd_vote_counts")
+
+
+def sum_apply(x: torch.Tensor, counts: torch.Tensor, M: int, d: int, ldc: int, delta: float,
+              stream=None) -> None:
+    """Worker side of the "(good)" scheme: x <- x - delta * (sum of the M signs), in place."""
+    _need(x, d, "x"); _need(counts, count_planes(M) * ldc, "counts")
+    _check(lib().ssgd_sum_apply(_ptr(x, torch.float32, "x"), _ptr(counts, WORD_DTYPE, "counts"), M, d,
+                                ldc, delta, _stream(stream)), "ssgd_sum_apply")
 
 
 def signsgd_step_host(x: torch.Tensor, g_host: torch.Tensor, m: Optional[torch.Tensor], M: int,

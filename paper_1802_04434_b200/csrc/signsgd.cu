@@ -73,6 +73,16 @@ __device__ __forceinline__ unsigned assemble_word(unsigned nibble, unsigned lane
 // lane group j = lane / 8.
 constexpr int kThreads = 256;
 
+// What a worker sends, and whether it keeps a momentum:
+//   kSignSGD       bit = sign(g)                       (Algorithm 1 / Algorithm 3 as printed)
+//   kSignum        m <- beta m + (1-beta) g, bit = sign(m)            (Algorithm 2)
+//   kSignumWarmup  m updated as in kSignum, bit = sign(g): the first C(beta)
+//                  iterations of Theorem 3, which accumulate the momentum as
+//                  normal but step with the sign of the stochastic gradient
+constexpr int kSignSGD = 0;
+constexpr int kSignum = 1;
+constexpr int kSignumWarmup = 2;
+
 // Within a group of eight lanes all lanes hold the same assembled word.  Lane
 // (lane % 8) == u keeps the word of unroll step u ("its" word), so that after the
 // UNROLL steps the 4 * UNROLL words of the span sit in 4 * UNROLL distinct lanes
@@ -86,13 +96,15 @@ __device__ __forceinline__ unsigned long long own_word_index(unsigned lane) {
 // worker kernel: [momentum update +] sign + 1-bit pack, all M rows in one launch.
 // Tiles are numbered row-major over (row, tile in row), one tile per CTA.
 
-template <bool MOMENTUM, int UNROLL>
+template <int MODE, int UNROLL>
 __global__ void __launch_bounds__(kThreads)
 worker_pack_kernel(const float* __restrict__ g, float* __restrict__ m,
                    uint32_t* __restrict__ bits, unsigned long long d,
                    unsigned long long ld, unsigned long long ldw,
                    unsigned long long tiles_per_row, unsigned long long total_tiles,
                    float beta, float omb) {
+  constexpr bool MOMENTUM = MODE != kSignSGD;
+  constexpr bool SIGN_OF_G = MODE != kSignum;
   constexpr unsigned long long TILE = (unsigned long long)kThreads * 4 * UNROLL;
   constexpr unsigned SPAN = 128 * UNROLL;
   const unsigned lane = threadIdx.x & 31u;
@@ -125,7 +137,7 @@ worker_pack_kernel(const float* __restrict__ g, float* __restrict__ m,
           v = momentum_update4(beta, omb, mv[u], v);
           st128(mr + e0 + u * 128 + lane * 4, v);
         }
-        const unsigned word = assemble_word(sign_nibble(v), lane);
+        const unsigned word = assemble_word(sign_nibble(SIGN_OF_G ? gv[u] : v), lane);
         if ((lane & 7u) == (unsigned)u) mine = word;
       }
       if ((lane & 7u) < (unsigned)UNROLL) br[own_word_index<UNROLL>(lane)] = mine;
@@ -139,12 +151,13 @@ worker_pack_kernel(const float* __restrict__ g, float* __restrict__ m,
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
           if (e + k < d) {
-            float v = gr[e + k];
+            const float gk = gr[e + k];
+            float v = gk;
             if (MOMENTUM) {
-              v = momentum_update(beta, omb, mr[e + k], v);
+              v = momentum_update(beta, omb, mr[e + k], gk);
               mr[e + k] = v;
             }
-            nib |= sign_bit(v) << k;
+            nib |= sign_bit(SIGN_OF_G ? gk : v) << k;
           }
         }
         const unsigned word = assemble_word(nib, lane);
@@ -256,13 +269,39 @@ struct Counter1 {
   __device__ __forceinline__ unsigned top() const { return c[NP - 1]; }
 };
 
+// Four words of one output plane; bits at positions >= d are written as 0,
+// whatever the rows held there, and words at or beyond ceil(d/32) are not written.
+__device__ __forceinline__ void store_plane_words(uint32_t* __restrict__ out, unsigned long long q,
+                                                  unsigned long long d, const W4& v) {
+  const unsigned long long first = q * 128;  // first parameter of this chunk
+  if (first + 128 <= d) {
+    *reinterpret_cast<uint4*>(out + 4 * q) = make_uint4(v.x, v.y, v.z, v.w);
+  } else {
+    const unsigned w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const unsigned long long lo = first + 32ull * k;
+      if (lo < d) {
+        const unsigned long long left = d - lo;
+        const unsigned mask = left >= 32 ? 0xFFFFFFFFu : ((1u << left) - 1u);
+        out[4 * q + k] = w[k] & mask;
+      }
+    }
+  }
+}
+
 // One thread owns four consecutive words (one 128-bit load per row) and walks
 // down the M rows; one 256-thread CTA covers 1024 words.
-template <int NP>
+//   COUNTS = false: out[W] receives the top plane, the voted bit (Algorithm 3).
+//   COUNTS = true:  the counter starts at 0 and all NP planes are written,
+//                   plane p at out + p * ldc: the number of +1 votes per parameter,
+//                   bit-sliced, which is what the server sends back in the "(good)"
+//                   scheme of Section 4.
+template <int NP, bool COUNTS>
 __global__ void __launch_bounds__(kThreads)
 vote_kernel(const uint32_t* __restrict__ bits, unsigned M, unsigned long long d,
-            unsigned long long W, unsigned long long ldw, uint32_t* __restrict__ vote,
-            unsigned start_value) {
+            unsigned long long W, unsigned long long ldw, uint32_t* __restrict__ out,
+            unsigned long long ldc, unsigned start_value) {
   const unsigned long long chunks = (W + 3) / 4;
   const unsigned long long stride = (unsigned long long)gridDim.x * kThreads;
   for (unsigned long long q = (unsigned long long)blockIdx.x * kThreads + threadIdx.x;
@@ -300,22 +339,11 @@ vote_kernel(const uint32_t* __restrict__ bits, unsigned M, unsigned long long d,
       cnt.template add<0>(ld_words(col + (unsigned long long)w * ldw));
       w += 1;
     }
-    W4 v = cnt.c[NP - 1];
-    // bits at positions >= d are written as 0, whatever the rows held there
-    const unsigned long long first = q * 128;  // first parameter of this chunk
-    unsigned out[4] = {v.x, v.y, v.z, v.w};
-    if (first + 128 <= d) {
-      *reinterpret_cast<uint4*>(vote + 4 * q) = make_uint4(out[0], out[1], out[2], out[3]);
-    } else {
+    if (COUNTS) {
 #pragma unroll
-      for (int k = 0; k < 4; ++k) {
-        const unsigned long long lo = first + 32ull * k;
-        if (lo < d) {
-          const unsigned long long left = d - lo;
-          const unsigned mask = left >= 32 ? 0xFFFFFFFFu : ((1u << left) - 1u);
-          vote[4 * q + k] = out[k] & mask;
-        }
-      }
+      for (int p = 0; p < NP; ++p) store_plane_words(out + (unsigned long long)p * ldc, q, d, cnt.c[p]);
+    } else {
+      store_plane_words(out, q, d, cnt.c[NP - 1]);
     }
   }
 }
@@ -366,6 +394,47 @@ apply_kernel(float* __restrict__ x, const uint32_t* __restrict__ vote, unsigned 
 }
 
 // ---------------------------------------------------------------------------
+// sum-apply: the "(good)" update of Section 4, x <- x - delta * sum_m sign(.),
+// from the bit-sliced count P of +1 votes: the sum of signs is 2P - M.  One fused
+// multiply-add per element, x <- fma(-delta, float(2P - M), x).  Lane layout as
+// in the apply kernel; each lane reads its word of every count plane.
+
+template <int NP>
+__global__ void __launch_bounds__(kThreads)
+sum_apply_kernel(float* __restrict__ x, const uint32_t* __restrict__ counts, unsigned M,
+                 unsigned long long d, unsigned long long ldc, float delta) {
+  const unsigned lane = threadIdx.x & 31u;
+  const unsigned long long stride = (unsigned long long)gridDim.x * kThreads * 4;
+  const float neg = -delta;
+  for (unsigned long long e = ((unsigned long long)blockIdx.x * kThreads + threadIdx.x) * 4; e < d; e += stride) {
+    const unsigned shift = 4u * (lane & 7u);        // e is a multiple of 4: (e % 32) = 4 (lane % 8)
+    unsigned nib[NP];
+#pragma unroll
+    for (int p = 0; p < NP; ++p) nib[p] = __ldg(counts + (unsigned long long)p * ldc + (e >> 5)) >> shift;
+    float s[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      int P = 0;
+#pragma unroll
+      for (int p = 0; p < NP; ++p) P |= (int)((nib[p] >> k) & 1u) << p;
+      s[k] = (float)(2 * P - (int)M);
+    }
+    if (e + 4 <= d) {
+      float4 v = ld128(x + e);
+      v.x = __fmaf_rn(neg, s[0], v.x);
+      v.y = __fmaf_rn(neg, s[1], v.y);
+      v.z = __fmaf_rn(neg, s[2], v.z);
+      v.w = __fmaf_rn(neg, s[3], v.w);
+      st128(x + e, v);
+    } else {
+#pragma unroll
+      for (int k = 0; k < 4; ++k)
+        if (e + k < d) x[e + k] = __fmaf_rn(neg, s[k], x[e + k]);
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------
 // fused step: one launch does the worker step for all M rows, the vote and the
 // apply on a tile of columns, so that the sign words are never read back from
 // memory and x is touched by the CTA that voted on it.  Per parameter it moves
@@ -387,11 +456,13 @@ apply_kernel(float* __restrict__ x, const uint32_t* __restrict__ vote, unsigned 
 constexpr int kFusedMaxWorkers = 8;   // rows walked by one CTA at most
 constexpr int kFusedMaxPlanes = 4;    // planes needed for M <= 8
 
-template <bool MOMENTUM, int UNROLL, int NP>
+template <int MODE, int UNROLL, int NP>
 __device__ __forceinline__ void fused_row(const float* __restrict__ gr, float* __restrict__ mr,
                                           uint32_t* __restrict__ brow, float beta, float omb,
                                           unsigned lane, unsigned sub, unsigned long long my_word,
                                           Counter1<NP>& cnt) {
+  constexpr bool MOMENTUM = MODE != kSignSGD;
+  constexpr bool SIGN_OF_G = MODE != kSignum;
   float4 gv[UNROLL], mv[UNROLL];
 #pragma unroll
   for (int u = 0; u < UNROLL; ++u) gv[u] = ld128(gr + u * 128);
@@ -407,7 +478,7 @@ __device__ __forceinline__ void fused_row(const float* __restrict__ gr, float* _
       v = momentum_update4(beta, omb, mv[u], v);
       st128(mr + u * 128, v);
     }
-    const unsigned word = assemble_word(sign_nibble(v), lane);
+    const unsigned word = assemble_word(sign_nibble(SIGN_OF_G ? gv[u] : v), lane);
     if (sub == (unsigned)u) mine = word;
   }
   if (sub < (unsigned)UNROLL) brow[my_word] = mine;
@@ -418,13 +489,15 @@ __device__ __forceinline__ void fused_row(const float* __restrict__ gr, float* _
 // guards.  Bits at positions >= d stay 0 in every row, so they count 0 votes and
 // the voted word has them 0 as well (the threshold is at least 1).  Kept out of
 // line so that the interior path's register allocation is not affected.
-template <bool MOMENTUM, int UNROLL, int NP>
+template <int MODE, int UNROLL, int NP>
 __device__ __noinline__ void fused_ragged_span(const float* __restrict__ g, float* __restrict__ m,
                                                float* __restrict__ x, uint32_t* __restrict__ bits,
                                                uint32_t* __restrict__ vote, unsigned M,
                                                unsigned long long d, unsigned long long ld,
                                                unsigned long long ldw, float beta, float omb, float delta,
                                                unsigned start_value, unsigned long long e0) {
+  constexpr bool MOMENTUM = MODE != kSignSGD;
+  constexpr bool SIGN_OF_G = MODE != kSignum;
   const unsigned lane = threadIdx.x & 31u;
   const unsigned sub = lane & 7u;
   const float minus = -delta;
@@ -443,12 +516,13 @@ __device__ __noinline__ void fused_ragged_span(const float* __restrict__ g, floa
 #pragma unroll
       for (int k = 0; k < 4; ++k) {
         if (e + k < d) {
-          float v = gr[e + k];
+          const float gk = gr[e + k];
+          float v = gk;
           if (MOMENTUM) {
-            v = momentum_update(beta, omb, mr[e + k], v);
+            v = momentum_update(beta, omb, mr[e + k], gk);
             mr[e + k] = v;
           }
-          nib |= sign_bit(v) << k;
+          nib |= sign_bit(SIGN_OF_G ? gk : v) << k;
         }
       }
       const unsigned word = assemble_word(nib, lane);
@@ -470,12 +544,13 @@ __device__ __noinline__ void fused_ragged_span(const float* __restrict__ g, floa
   }
 }
 
-template <bool MOMENTUM, int UNROLL, int NP>
+template <int MODE, int UNROLL, int NP>
 __global__ void __launch_bounds__(kThreads, 5)
 fused_step_kernel(const float* __restrict__ g, float* __restrict__ m, float* __restrict__ x,
                   uint32_t* __restrict__ bits, uint32_t* __restrict__ vote, unsigned M,
                   unsigned long long d, unsigned long long ld, unsigned long long ldw,
                   float beta, float omb, float delta, unsigned start_value) {
+  constexpr bool MOMENTUM = MODE != kSignSGD;
   constexpr unsigned long long TILE = (unsigned long long)kThreads * 4 * UNROLL;
   constexpr unsigned SPAN = 128 * UNROLL;
   const unsigned lane = threadIdx.x & 31u;
@@ -484,7 +559,7 @@ fused_step_kernel(const float* __restrict__ g, float* __restrict__ m, float* __r
   const unsigned long long e0 = (unsigned long long)blockIdx.x * TILE + (unsigned long long)warp * SPAN;
   if (e0 >= d) return;   // uniform over the warp; nothing below synchronises across warps
   if (e0 + SPAN > d) {
-    fused_ragged_span<MOMENTUM, UNROLL, NP>(g, m, x, bits, vote, M, d, ld, ldw, beta, omb, delta,
+    fused_ragged_span<MODE, UNROLL, NP>(g, m, x, bits, vote, M, d, ld, ldw, beta, omb, delta,
                                             start_value, e0);
     return;
   }
@@ -493,7 +568,7 @@ fused_step_kernel(const float* __restrict__ g, float* __restrict__ m, float* __r
   const unsigned long long my_word = (e0 >> 5) + own_word_index<UNROLL>(lane);
   const unsigned long long off = e0 + lane * 4;
   for (unsigned row = 0; row < M; ++row) {
-    fused_row<MOMENTUM, UNROLL, NP>(g + (unsigned long long)row * ld + off,
+    fused_row<MODE, UNROLL, NP>(g + (unsigned long long)row * ld + off,
                                     MOMENTUM ? m + (unsigned long long)row * ld + off : nullptr,
                                     bits + (unsigned long long)row * ldw, beta, omb, lane, sub, my_word, cnt);
   }
@@ -569,26 +644,26 @@ int pick_unroll(unsigned long long elements_per_row, unsigned long long rows, in
   return 1;
 }
 
-template <bool MOMENTUM, int UNROLL>
+template <int MODE, int UNROLL>
 void launch_worker_u(const float* g, float* m, size_t M, size_t d, size_t ld, float beta,
                      uint32_t* bits, size_t ldw, cudaStream_t s) {
   constexpr unsigned long long TILE = (unsigned long long)kThreads * 4 * UNROLL;
   const unsigned long long tiles_per_row = (d + TILE - 1) / TILE;
   const unsigned long long total = tiles_per_row * M;
   const float omb = 1.0f - beta;
-  worker_pack_kernel<MOMENTUM, UNROLL><<<grid_for(total), kThreads, 0, s>>>(
+  worker_pack_kernel<MODE, UNROLL><<<grid_for(total), kThreads, 0, s>>>(
       g, m, bits, d, ld, ldw, tiles_per_row, total, beta, omb);
 }
 
-template <bool MOMENTUM>
+template <int MODE>
 ssgd_status launch_worker(const float* g, float* m, size_t M, size_t d, size_t ld, float beta,
                           uint32_t* bits, size_t ldw, cudaStream_t s) {
   DeviceInfo di;
   if (!device_info(&di)) return SSGD_ERR_CUDA;
   switch (pick_unroll(d, M, di.sms)) {
-    case 4: launch_worker_u<MOMENTUM, 4>(g, m, M, d, ld, beta, bits, ldw, s); break;
-    case 2: launch_worker_u<MOMENTUM, 2>(g, m, M, d, ld, beta, bits, ldw, s); break;
-    default: launch_worker_u<MOMENTUM, 1>(g, m, M, d, ld, beta, bits, ldw, s); break;
+    case 4: launch_worker_u<MODE, 4>(g, m, M, d, ld, beta, bits, ldw, s); break;
+    case 2: launch_worker_u<MODE, 2>(g, m, M, d, ld, beta, bits, ldw, s); break;
+    default: launch_worker_u<MODE, 1>(g, m, M, d, ld, beta, bits, ldw, s); break;
   }
   return launch_status();
 }
@@ -604,29 +679,69 @@ unsigned vote_start_value(size_t M, unsigned planes) {
   return (1u << (planes - 1)) - (unsigned)((M + 1) / 2);
 }
 
-template <int NP>
-void launch_vote_np(const uint32_t* bits, size_t M, size_t d, size_t W, size_t ldw, uint32_t* vote,
-                    unsigned grid, cudaStream_t s) {
-  vote_kernel<NP><<<grid, kThreads, 0, s>>>(bits, (unsigned)M, d, W, ldw, vote, vote_start_value(M, NP));
+template <int NP, bool COUNTS>
+void launch_vote_np(const uint32_t* bits, size_t M, size_t d, size_t W, size_t ldw, uint32_t* out,
+                    size_t ldc, unsigned grid, cudaStream_t s) {
+  const unsigned start = COUNTS ? 0u : vote_start_value(M, NP);
+  vote_kernel<NP, COUNTS><<<grid, kThreads, 0, s>>>(bits, (unsigned)M, d, W, ldw, out, ldc, start);
+}
+
+// planes that hold a count in 0..M: the bit length of M
+unsigned count_planes(size_t M) {
+  unsigned n = 0;
+  while ((M >> n) != 0) ++n;
+  return n;
+}
+
+template <bool COUNTS>
+ssgd_status launch_vote_any(const uint32_t* bits, size_t M, size_t d, size_t ldw, uint32_t* out,
+                            size_t ldc, cudaStream_t s) {
+  const size_t W = ssgd_words(d);
+  const unsigned long long chunks = (W + 3) / 4;
+  const unsigned grid = grid_for((chunks + kThreads - 1) / kThreads);
+  switch (COUNTS ? count_planes(M) : vote_planes(M)) {
+    case 1: launch_vote_np<1, COUNTS>(bits, M, d, W, ldw, out, ldc, grid, s); break;
+    case 2: launch_vote_np<2, COUNTS>(bits, M, d, W, ldw, out, ldc, grid, s); break;
+    case 3: launch_vote_np<3, COUNTS>(bits, M, d, W, ldw, out, ldc, grid, s); break;
+    case 4: launch_vote_np<4, COUNTS>(bits, M, d, W, ldw, out, ldc, grid, s); break;
+    case 5: launch_vote_np<5, COUNTS>(bits, M, d, W, ldw, out, ldc, grid, s); break;
+    case 6: launch_vote_np<6, COUNTS>(bits, M, d, W, ldw, out, ldc, grid, s); break;
+    case 7: launch_vote_np<7, COUNTS>(bits, M, d, W, ldw, out, ldc, grid, s); break;
+    case 8: launch_vote_np<8, COUNTS>(bits, M, d, W, ldw, out, ldc, grid, s); break;
+    case 9: launch_vote_np<9, COUNTS>(bits, M, d, W, ldw, out, ldc, grid, s); break;
+    case 10: launch_vote_np<10, COUNTS>(bits, M, d, W, ldw, out, ldc, grid, s); break;
+    case 11: launch_vote_np<11, COUNTS>(bits, M, d, W, ldw, out, ldc, grid, s); break;
+    default: return SSGD_ERR_SIZE;
+  }
+  return launch_status();
 }
 
 ssgd_status launch_vote(const uint32_t* bits, size_t M, size_t d, size_t ldw, uint32_t* vote,
                         cudaStream_t s) {
-  const size_t W = ssgd_words(d);
-  const unsigned long long chunks = (W + 3) / 4;
-  const unsigned grid = grid_for((chunks + kThreads - 1) / kThreads);
-  switch (vote_planes(M)) {
-    case 1: launch_vote_np<1>(bits, M, d, W, ldw, vote, grid, s); break;
-    case 2: launch_vote_np<2>(bits, M, d, W, ldw, vote, grid, s); break;
-    case 3: launch_vote_np<3>(bits, M, d, W, ldw, vote, grid, s); break;
-    case 4: launch_vote_np<4>(bits, M, d, W, ldw, vote, grid, s); break;
-    case 5: launch_vote_np<5>(bits, M, d, W, ldw, vote, grid, s); break;
-    case 6: launch_vote_np<6>(bits, M, d, W, ldw, vote, grid, s); break;
-    case 7: launch_vote_np<7>(bits, M, d, W, ldw, vote, grid, s); break;
-    case 8: launch_vote_np<8>(bits, M, d, W, ldw, vote, grid, s); break;
-    case 9: launch_vote_np<9>(bits, M, d, W, ldw, vote, grid, s); break;
-    case 10: launch_vote_np<10>(bits, M, d, W, ldw, vote, grid, s); break;
-    case 11: launch_vote_np<11>(bits, M, d, W, ldw, vote, grid, s); break;
+  return launch_vote_any<false>(bits, M, d, ldw, vote, 0, s);
+}
+
+template <int NP>
+void launch_sum_apply_np(float* x, const uint32_t* counts, size_t M, size_t d, size_t ldc, float delta,
+                         cudaStream_t s) {
+  const unsigned long long ctas = ((d + 3) / 4 + kThreads - 1) / kThreads;
+  sum_apply_kernel<NP><<<grid_for(ctas), kThreads, 0, s>>>(x, counts, (unsigned)M, d, ldc, delta);
+}
+
+ssgd_status launch_sum_apply(float* x, const uint32_t* counts, size_t M, size_t d, size_t ldc,
+                             float delta, cudaStream_t s) {
+  switch (count_planes(M)) {
+    case 1: launch_sum_apply_np<1>(x, counts, M, d, ldc, delta, s); break;
+    case 2: launch_sum_apply_np<2>(x, counts, M, d, ldc, delta, s); break;
+    case 3: launch_sum_apply_np<3>(x, counts, M, d, ldc, delta, s); break;
+    case 4: launch_sum_apply_np<4>(x, counts, M, d, ldc, delta, s); break;
+    case 5: launch_sum_apply_np<5>(x, counts, M, d, ldc, delta, s); break;
+    case 6: launch_sum_apply_np<6>(x, counts, M, d, ldc, delta, s); break;
+    case 7: launch_sum_apply_np<7>(x, counts, M, d, ldc, delta, s); break;
+    case 8: launch_sum_apply_np<8>(x, counts, M, d, ldc, delta, s); break;
+    case 9: launch_sum_apply_np<9>(x, counts, M, d, ldc, delta, s); break;
+    case 10: launch_sum_apply_np<10>(x, counts, M, d, ldc, delta, s); break;
+    case 11: launch_sum_apply_np<11>(x, counts, M, d, ldc, delta, s); break;
     default: return SSGD_ERR_SIZE;
   }
   return launch_status();
@@ -660,29 +775,29 @@ struct StepArgs {
   float beta, delta;
 };
 
-template <bool MOMENTUM, int UNROLL, int NP>
+template <int MODE, int UNROLL, int NP>
 void launch_fused_mun(const StepArgs& a, cudaStream_t s) {
   constexpr unsigned long long TILE = (unsigned long long)kThreads * 4 * UNROLL;
   const unsigned long long tiles = (a.d + TILE - 1) / TILE;
-  fused_step_kernel<MOMENTUM, UNROLL, NP><<<(unsigned)tiles, kThreads, 0, s>>>(
+  fused_step_kernel<MODE, UNROLL, NP><<<(unsigned)tiles, kThreads, 0, s>>>(
       a.g, a.m, a.x, a.bits, a.vote, (unsigned)a.M, a.d, a.ld, a.ldw, a.beta, 1.0f - a.beta, a.delta,
       vote_start_value(a.M, NP));
 }
 
-template <bool MOMENTUM, int UNROLL>
+template <int MODE, int UNROLL>
 bool launch_fused_mu(const StepArgs& a, cudaStream_t s) {
   switch (vote_planes(a.M)) {
-    case 1: launch_fused_mun<MOMENTUM, UNROLL, 1>(a, s); return true;
-    case 2: launch_fused_mun<MOMENTUM, UNROLL, 2>(a, s); return true;
-    case 3: launch_fused_mun<MOMENTUM, UNROLL, 3>(a, s); return true;
-    case 4: launch_fused_mun<MOMENTUM, UNROLL, 4>(a, s); return true;
+    case 1: launch_fused_mun<MODE, UNROLL, 1>(a, s); return true;
+    case 2: launch_fused_mun<MODE, UNROLL, 2>(a, s); return true;
+    case 3: launch_fused_mun<MODE, UNROLL, 3>(a, s); return true;
+    case 4: launch_fused_mun<MODE, UNROLL, 4>(a, s); return true;
   }
   return false;
 }
 
 // Whether the step runs as the fused kernel: few workers, and a vector that fits
 // one grid of tiles.  Everything else takes the three kernels.
-template <bool MOMENTUM>
+template <int MODE>
 ssgd_status launch_fused(const StepArgs& a, cudaStream_t s, bool* launched) {
   static_assert(kFusedMaxWorkers / 2 < (1 << (kFusedMaxPlanes - 1)), "planes cover the fused worker limit");
   *launched = false;
@@ -692,10 +807,24 @@ ssgd_status launch_fused(const StepArgs& a, cudaStream_t s, bool* launched) {
   const int unroll = pick_unroll(a.d, 1, di.sms) >= 2 ? 2 : 1;
   const unsigned long long tile = (unsigned long long)kThreads * 4 * unroll;
   if ((a.d + tile - 1) / tile > kMaxGrid) return SSGD_OK;
-  const bool ok = unroll == 2 ? launch_fused_mu<MOMENTUM, 2>(a, s) : launch_fused_mu<MOMENTUM, 1>(a, s);
+  const bool ok = unroll == 2 ? launch_fused_mu<MODE, 2>(a, s) : launch_fused_mu<MODE, 1>(a, s);
   if (!ok) return SSGD_ERR_SIZE;
   *launched = true;
   return launch_status();
+}
+
+// One whole step in the given worker mode: the fused kernel where it applies,
+// otherwise worker, vote and apply kernels on the same stream.
+template <int MODE>
+ssgd_status run_step(const StepArgs& a, cudaStream_t s) {
+  bool launched = false;
+  ssgd_status st = launch_fused<MODE>(a, s, &launched);
+  if (st != SSGD_OK || launched) return st;
+  st = launch_worker<MODE>(a.g, a.m, a.M, a.d, a.ld, a.beta, a.bits, a.ldw, s);
+  if (st != SSGD_OK) return st;
+  st = launch_vote(a.bits, a.M, a.d, a.ldw, a.vote, s);
+  if (st != SSGD_OK) return st;
+  return launch_apply(a.x, a.vote, a.d, a.delta, s);
 }
 
 // argument checks shared by the entry points -------------------------------
@@ -769,14 +898,14 @@ ssgd_status ssgd_sign_pack(const float* g, size_t M, size_t d, size_t ld, uint32
                            size_t ldw, void* stream) {
   const ssgd_status st = check_sign_pack(g, M, d, ld, bits, ldw);
   if (st != SSGD_OK || d == 0) return st;
-  return launch_worker<false>(g, nullptr, M, d, ld, 0.0f, bits, ldw, static_cast<cudaStream_t>(stream));
+  return launch_worker<kSignSGD>(g, nullptr, M, d, ld, 0.0f, bits, ldw, static_cast<cudaStream_t>(stream));
 }
 
 ssgd_status ssgd_signum_momentum_pack(const float* g, float* m, size_t M, size_t d, size_t ld,
                                       float beta, uint32_t* bits, size_t ldw, void* stream) {
   const ssgd_status st = check_momentum_pack(g, m, M, d, ld, beta, bits, ldw);
   if (st != SSGD_OK || d == 0) return st;
-  return launch_worker<true>(g, m, M, d, ld, beta, bits, ldw, static_cast<cudaStream_t>(stream));
+  return launch_worker<kSignum>(g, m, M, d, ld, beta, bits, ldw, static_cast<cudaStream_t>(stream));
 }
 
 ssgd_status ssgd_majority_vote(const uint32_t* bits, size_t M, size_t d, size_t ldw,
@@ -795,20 +924,66 @@ ssgd_status ssgd_sign_apply(float* x, const uint32_t* vote, size_t d, float delt
 ssgd_status ssgd_signsgd_step(float* x, const float* g, float* m, size_t M, size_t d, size_t ld,
                               float beta, float delta, uint32_t* bits_ws, size_t ldw,
                               uint32_t* vote_ws, void* stream) {
-  ssgd_status st = check_step(x, g, m, M, d, ld, beta, delta, bits_ws, ldw, vote_ws);
+  const ssgd_status st = check_step(x, g, m, M, d, ld, beta, delta, bits_ws, ldw, vote_ws);
   if (st != SSGD_OK || d == 0) return st;
-  cudaStream_t s = static_cast<cudaStream_t>(stream);
   const StepArgs a{g, m, x, bits_ws, vote_ws, M, d, ld, ldw, beta, delta};
-  bool launched = false;
-  st = m ? launch_fused<true>(a, s, &launched) : launch_fused<false>(a, s, &launched);
-  if (st != SSGD_OK || launched) return st;
-  // many workers, or a vector beyond one grid of tiles: the same step as three launches
-  st = m ? launch_worker<true>(g, m, M, d, ld, beta, bits_ws, ldw, s)
-         : launch_worker<false>(g, nullptr, M, d, ld, 0.0f, bits_ws, ldw, s);
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  return m ? run_step<kSignum>(a, s) : run_step<kSignSGD>(a, s);
+}
+
+size_t ssgd_warmup_steps(float beta) {
+  if (!beta_ok(beta)) return 0;
+  // C(beta) of Theorem 3: the least positive integer C with
+  //   (C / 2) beta^C <= 1 / ((1 - beta^2) (C + 1))   and   beta^(C + 1) <= 1 / 2.
+  const double b = (double)beta;
+  const double rhs = 1.0 / (1.0 - b * b);
+  double bc = b;  // beta^C
+  for (size_t C = 1; C != 0; ++C, bc *= b) {
+    if (0.5 * (double)C * bc * ((double)C + 1.0) <= rhs && bc * b <= 0.5) return C;
+  }
+  return 0;
+}
+
+ssgd_status ssgd_signum_warmup_pack(const float* g, float* m, size_t M, size_t d, size_t ld,
+                                    float beta, uint32_t* bits, size_t ldw, void* stream) {
+  const ssgd_status st = check_momentum_pack(g, m, M, d, ld, beta, bits, ldw);
+  if (st != SSGD_OK || d == 0) return st;
+  return launch_worker<kSignumWarmup>(g, m, M, d, ld, beta, bits, ldw, static_cast<cudaStream_t>(stream));
+}
+
+ssgd_status ssgd_signsgd_warmup_step(float* x, const float* g, float* m, size_t M, size_t d,
+                                     size_t ld, float beta, float delta, uint32_t* bits_ws,
+                                     size_t ldw, uint32_t* vote_ws, void* stream) {
+  if (!m) return SSGD_ERR_NULL;
+  const ssgd_status st = check_step(x, g, m, M, d, ld, beta, delta, bits_ws, ldw, vote_ws);
+  if (st != SSGD_OK || d == 0) return st;
+  const StepArgs a{g, m, x, bits_ws, vote_ws, M, d, ld, ldw, beta, delta};
+  return run_step<kSignumWarmup>(a, static_cast<cudaStream_t>(stream));
+}
+
+size_t ssgd_count_planes(size_t M) { return (M >= 1 && M <= SSGD_MAX_WORKERS) ? count_planes(M) : 0; }
+
+ssgd_status ssgd_vote_counts(const uint32_t* bits, size_t M, size_t d, size_t ldw, uint32_t* counts,
+                             size_t ldc, void* stream) {
+  if (!bits || !counts) return SSGD_ERR_NULL;
+  if (!aligned16(bits) || !aligned16(counts)) return SSGD_ERR_ALIGN;
+  ssgd_status st = check_rows(M, d, 0, ldw, false);
   if (st != SSGD_OK) return st;
-  st = launch_vote(bits_ws, M, d, ldw, vote_ws, s);
+  st = check_rows(count_planes(M), d, 0, ldc, false);   // the planes are rows of the same kind
+  if (st != SSGD_OK || d == 0) return st;
+  return launch_vote_any<true>(bits, M, d, ldw, counts, ldc, static_cast<cudaStream_t>(stream));
+}
+
+ssgd_status ssgd_sum_apply(float* x, const uint32_t* counts, size_t M, size_t d, size_t ldc,
+                           float delta, void* stream) {
+  if (!x || !counts) return SSGD_ERR_NULL;
+  if (!aligned16(x) || !aligned16(counts)) return SSGD_ERR_ALIGN;
+  if (M < 1 || M > SSGD_MAX_WORKERS) return SSGD_ERR_SIZE;
+  const ssgd_status st = check_rows(count_planes(M), d, 0, ldc, false);
   if (st != SSGD_OK) return st;
-  return launch_apply(x, vote_ws, d, delta, s);
+  if (!isfinite(delta)) return SSGD_ERR_ARG;
+  if (d == 0) return SSGD_OK;
+  return launch_sum_apply(x, counts, M, d, ldc, delta, static_cast<cudaStream_t>(stream));
 }
 
 ssgd_status ssgd_signsgd_step_host(float* x, const float* g_host, float* m, size_t M, size_t d,

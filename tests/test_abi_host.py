@@ -108,6 +108,33 @@ def test_step_argument_checks(L):
     assert h(A, A, A, 1, 64, 64, 0.9, 0.1, A + 4, A, 4, A, None, None) == ALIGN
 
 
+def test_warmup_steps_is_host_arithmetic(L):
+    assert L.ssgd_warmup_steps(0.9) == 54          # Theorem 3: "for beta = 0.9 we have C = 54"
+    assert L.ssgd_warmup_steps(0.0) == 1
+    assert L.ssgd_warmup_steps(1.0) == 0 and L.ssgd_warmup_steps(float("nan")) == 0
+    w = L.ssgd_signsgd_warmup_step
+    assert w(A, A, None, 1, 64, 64, 0.9, 0.1, A, 4, A, None) == NULL     # m is required
+    assert w(A, A, A, 1, 0, 0, 0.9, 0.1, A, 0, A, None) == OK
+    assert L.ssgd_signum_warmup_pack(A, A, 1, 64, 64, 1.0, A, 4, None) == ARG
+
+
+def test_good_scheme_argument_checks(L):
+    assert [L.ssgd_count_planes(M) for M in (1, 2, 3, 4, 7, 8, 1024)] == [1, 2, 2, 3, 3, 4, 11]
+    assert L.ssgd_count_planes(0) == 0 and L.ssgd_count_planes(1025) == 0
+    c = L.ssgd_vote_counts
+    assert c(None, 3, 64, 4, A, 4, None) == NULL
+    assert c(A, 3, 64, 4, A + 4, 4, None) == ALIGN
+    assert c(A, 3, 64, 4, A, 2, None) == ALIGN
+    assert c(A, 3, 640, 20, A, 16, None) == SIZE            # ldc < W
+    assert c(A, 0, 64, 4, A, 4, None) == SIZE
+    assert c(A, 3, 0, 0, A, 0, None) == OK
+    a = L.ssgd_sum_apply
+    assert a(None, A, 3, 64, 4, 0.1, None) == NULL
+    assert a(A, A, 0, 64, 4, 0.1, None) == SIZE
+    assert a(A, A, 3, 64, 4, float("inf"), None) == ARG
+    assert a(A, A, 3, 0, 0, 0.1, None) == OK
+
+
 def test_binding_refuses_to_run_without_the_library(monkeypatch, tmp_path):
     from paper_1802_04434_b200 import binding
     monkeypatch.setattr(binding, "_lib", None)

@@ -340,3 +340,94 @@ def test_resume_from_copied_state_is_bit_identical():
     for k in range(2, 5):
         B.signsgd_step(xb, gs[k], mb, M, d, ld, cfg.beta, cfg.delta, bits, ldw, vote)
     assert torch.equal(xa, xb) and torch.equal(ma, mb)
+
+
+# ------------------------------------------------------------------ Theorem 3 warm-up
+
+def test_warmup_length_matches_oracle():
+    for beta in (0.0, 0.3, 0.5, 0.8, 0.9, 0.95, 0.99, 0.999):
+        assert B.warmup_steps(beta) == oracle.warmup_steps(beta)
+    assert B.warmup_steps(0.9) == 54
+    assert B.warmup_steps(1.0) == 0 and B.warmup_steps(float("nan")) == 0
+
+
+@pytest.mark.parametrize("M,d", [(1, 1000), (3, 4097), (7, 100003), (8, 1 << 20), (16, 70001), (33, 5000)])
+def test_warmup_pack_and_step(M, d):
+    ld, W = wl.round_up(d, 4), oracle.words(d)
+    ldw = wl.round_up(W, 4)
+    g, m, x = rand_inputs(M, d, ld, seed=M + d, special=True)
+    with np.errstate(over="ignore"):
+        m *= 3.0
+    gd, md = torch.from_numpy(g).to(DEV), torch.from_numpy(m).to(DEV)
+    bits = torch.zeros(M, ldw, dtype=torch.int32, device=DEV)
+    B.signum_warmup_pack(gd, md, M, d, ld, 0.9, bits, ldw)
+    m_ref = m.copy().reshape(-1)
+    b_ref = oracle.signum_warmup_pack(g.reshape(-1), m_ref, M, d, 0.9, ld=ld, ldw=ldw)
+    assert np.array_equal(u32(bits).reshape(-1), b_ref)
+    assert_same_f32(f32(md).reshape(-1), m_ref, "m")
+    # whole step
+    md, xd = torch.from_numpy(m).to(DEV), torch.from_numpy(x).to(DEV)
+    vote = torch.zeros(W, dtype=torch.int32, device=DEV)
+    B.signsgd_warmup_step(xd, gd, md, M, d, ld, 0.9, 1e-3, bits, ldw, vote)
+    m_ref, x_ref = m.copy().reshape(-1), x.copy()
+    b_ref, v_ref = oracle.signsgd_warmup_step(x_ref, g.reshape(-1), m_ref, M, d, 0.9, 1e-3, ld=ld, ldw=ldw)
+    assert np.array_equal(u32(bits).reshape(-1), b_ref) and np.array_equal(u32(vote), v_ref)
+    assert_same_f32(f32(xd), x_ref, "x")
+    assert_same_f32(f32(md).reshape(-1), m_ref, "m")
+
+
+def test_warmup_then_signum_schedule():
+    """Theorem 3's schedule on the small workload: warm-up steps first, Signum steps after."""
+    cfg = wl.small_signum(d=100_000, M=3)
+    M, d, ld, ldw, W = cfg.M, cfg.d, cfg.ld, cfg.ldw, cfg.words
+    mu = cfg.shared(DEV)
+    xd, md = cfg.x0(DEV), cfg.m0(DEV)
+    x_ref, m_ref = f32(xd).copy(), f32(md).reshape(-1).copy()
+    bits = torch.zeros(M, ldw, dtype=torch.int32, device=DEV)
+    vote = torch.zeros(W, dtype=torch.int32, device=DEV)
+    C = 3                                      # a short warm-up keeps the test fast
+    for k in range(6):
+        gd = cfg.g(k, DEV, mu)
+        gh = f32(gd).reshape(-1)
+        if k < C:
+            B.signsgd_warmup_step(xd, gd, md, M, d, ld, cfg.beta, cfg.delta, bits, ldw, vote)
+            b_ref, v_ref = oracle.signsgd_warmup_step(x_ref, gh, m_ref, M, d, cfg.beta, cfg.delta, ld=ld, ldw=ldw)
+        else:
+            B.signsgd_step(xd, gd, md, M, d, ld, cfg.beta, cfg.delta, bits, ldw, vote)
+            b_ref, v_ref = oracle.signsgd_step(x_ref, gh, m_ref, M, d, cfg.beta, cfg.delta, ld=ld, ldw=ldw)
+        assert np.array_equal(u32(bits).reshape(-1), b_ref) and np.array_equal(u32(vote), v_ref)
+        assert_same_f32(f32(xd), x_ref, "x step %d" % k)
+        assert_same_f32(f32(md).reshape(-1), m_ref, "m step %d" % k)
+
+
+# ------------------------------------------------------------------ the "(good)" scheme of Sec. 4
+
+@pytest.mark.parametrize("M", [1, 2, 3, 7, 8, 15, 16, 31, 33, 255, 1024])
+def test_vote_counts_and_sum_apply(M):
+    for d in (1, 33, 1000, 4097, 100003 if M <= 33 else 5000):
+        r = np.random.default_rng(M * 7 + d)
+        W = oracle.words(d)
+        ldw, ldc = wl.round_up(W, 4), wl.round_up(W, 4) + 4
+        NPc = M.bit_length()
+        assert B.count_planes(M) == NPc
+        s = (r.random((M, d)) < r.random(d)).astype(np.uint8)
+        rows = np.zeros((M, ldw), dtype=np.uint32)
+        for w in range(M):
+            rows[w, :W] = oracle.pack_bits(s[w])
+        counts = torch.full((NPc, ldc), CANARY_WORD, dtype=torch.int32, device=DEV)
+        B.vote_counts(torch.from_numpy(rows.view(np.int32)).to(DEV), M, d, ldw, counts, ldc)
+        ref = oracle.vote_count_planes(rows.reshape(-1), M, d, ldw=ldw, ldc=ldc).reshape(NPc, ldc)
+        got = u32(counts)
+        assert np.array_equal(got[:, :W], ref[:, :W]), "M=%d d=%d" % (M, d)
+        assert np.all(got[:, W:] == np.uint32(0xDEADBEEF))
+        x = np.full(d + 5, CANARY_F, dtype=np.float32)
+        x[:d] = (r.standard_normal(d) * 10.0 ** r.integers(-4, 2, d)).astype(np.float32)
+        xd = torch.from_numpy(x).to(DEV)
+        clean = counts.clone()
+        clean[:, W:] = 0
+        B.sum_apply(xd, clean, M, d, ldc, 2e-3)
+        x_ref = x[:d].copy()
+        oracle.sum_apply(x_ref, ref.reshape(-1).copy(), M, d, 2e-3, ldc=ldc)
+        gx = f32(xd)
+        assert_same_f32(gx[:d], x_ref, "x (M=%d d=%d)" % (M, d))
+        assert np.all(gx[d:] == np.float32(CANARY_F))

@@ -415,3 +415,94 @@ def test_single_worker_algorithms_1_and_2():
     # m_new = 0.5 m + 0.5 g = [0.65, 0.4, -0.5, 0, -47.5]
     assert m.tolist() == [np.float32(0.65), np.float32(0.4), -0.5, 0.0, -47.5]
     assert x.tolist() == [-0.25, -0.25, 0.25, -0.25, 0.25]
+
+
+# ---------------------------------------------------------------- Theorem 3 warm-up
+
+def warmup_conditions(beta32, C):
+    """The two inequalities of Theorem 3's C(beta), in exact rational arithmetic."""
+    b = f32_to_fraction(beta32)
+    first = Fraction(C, 2) * b ** C <= 1 / (1 - b * b) * Fraction(1, C + 1)
+    second = b ** (C + 1) <= Fraction(1, 2)
+    return first, second
+
+
+def test_warmup_length_is_54_at_beta_0_9_as_printed():
+    assert oracle.warmup_steps(0.9) == int(GOLDEN["warmup_C_beta_0.9"]) == 54
+    b = np.float32(0.9)
+    assert warmup_conditions(b, 54) == (True, True)
+    assert warmup_conditions(b, 53)[0] is False          # 53 fails the first inequality
+    assert all(warmup_conditions(b, C) != (True, True) for C in range(1, 54))
+
+
+@pytest.mark.parametrize("beta", [0.0, 0.1, 0.5, 0.75, 0.8, 0.95, 0.99, 0.995])
+def test_warmup_length_is_the_least_integer_satisfying_both_conditions(beta):
+    b = np.float32(beta)
+    C = oracle.warmup_steps(float(b))
+    assert C >= 1 and warmup_conditions(b, C) == (True, True)
+    assert all(warmup_conditions(b, c) != (True, True) for c in range(1, C))
+
+
+def test_warmup_length_rejects_bad_beta():
+    for beta in (1.0, 1.5, -0.1, float("nan")):
+        assert oracle.warmup_steps(beta) == 0
+
+
+def test_warmup_pack_sends_sign_of_gradient_and_keeps_signum_momentum():
+    r = rng(51)
+    M, d = 4, 1500
+    g = r.standard_normal((M, d)).astype(np.float32).reshape(-1)
+    m0 = (r.standard_normal((M, d)) * 3).astype(np.float32).reshape(-1)   # momentum often disagrees with g
+    m_w, m_s = m0.copy(), m0.copy()
+    bits_w = oracle.signum_warmup_pack(g, m_w, M, d, 0.9)
+    bits_s = oracle.signum_momentum_pack(g, m_s, M, d, 0.9)
+    assert np.array_equal(m_w, m_s)                                       # momentum accumulates as normal
+    assert np.array_equal(bits_w, oracle.sign_pack(g, M, d))              # but the update uses sign(g)
+    assert not np.array_equal(bits_w, bits_s)
+    # whole step: x moves by the vote over sign(g)
+    x = r.standard_normal(d).astype(np.float32)
+    x1, m1 = x.copy(), m0.copy()
+    b1, v1 = oracle.signsgd_warmup_step(x1, g, m1, M, d, 0.9, 1e-3)
+    x2 = x.copy()
+    b2, v2 = oracle.signsgd_step(x2, g, None, M, d, 0.0, 1e-3)
+    assert np.array_equal(b1, b2) and np.array_equal(v1, v2) and np.array_equal(x1, x2)
+    assert np.array_equal(m1, m_s)
+
+
+# ---------------------------------------------------------------- the "(good)" scheme
+
+@pytest.mark.parametrize("M", [1, 2, 3, 4, 7, 8, 15, 16, 31, 32, 100, 1024])
+def test_count_planes_hold_the_integer_sum_of_signs(M):
+    r = rng(60 + M)
+    d = 500
+    assert oracle.count_planes(M) == M.bit_length()
+    s = (r.random((M, d)) < r.random(d)).astype(np.uint8)
+    bits = np.concatenate([np.array(py_pack(row.tolist()), dtype=np.uint32) for row in s])
+    planes = oracle.vote_count_planes(bits, M, d).reshape(M.bit_length(), -1)
+    P = s.sum(axis=0, dtype=np.int64)
+    for p in range(M.bit_length()):
+        assert planes[p].tolist() == py_pack(((P >> p) & 1).tolist())
+    # the sign of the sum is the majority vote, the tie (sum = 0) voting +1
+    vote = oracle.unpack_bits(oracle.majority_vote(bits, M, d), d)
+    assert np.array_equal(vote, (2 * P - M >= 0).astype(np.uint8))
+
+
+def test_sum_apply_is_x_minus_delta_times_sum_rounded_once():
+    r = rng(61)
+    M, d = 7, 600
+    s = r.integers(0, 2, size=(M, d), dtype=np.uint8)
+    bits = np.concatenate([np.array(py_pack(row.tolist()), dtype=np.uint32) for row in s])
+    planes = oracle.vote_count_planes(bits, M, d)
+    x = (r.standard_normal(d) * 10.0 ** r.integers(-5, 2, d)).astype(np.float32)
+    delta = np.float32(3e-3)
+    got = x.copy()
+    oracle.sum_apply(got, planes, M, d, float(delta))
+    S = 2 * s.sum(axis=0, dtype=np.int64) - M
+    expect = [round_f32(Fraction(xi) - Fraction(float(delta)) * int(si)) for xi, si in zip(x.tolist(), S.tolist())]
+    assert got.tolist() == expect
+    # M = 1: the sum of one sign is that sign, so the update is Algorithm 1's
+    one = oracle.vote_count_planes(bits[:oracle.words(d)].copy(), 1, d)
+    xa, xb = x.copy(), x.copy()
+    oracle.sum_apply(xa, one, 1, d, float(delta))
+    oracle.sign_apply(xb, bits[:oracle.words(d)].copy(), d, float(delta))
+    assert np.array_equal(xa, xb)
