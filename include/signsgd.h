@@ -159,6 +159,58 @@ ssgd_status ssgd_vote_counts(const uint32_t* bits, size_t M, size_t d, size_t ld
 ssgd_status ssgd_sum_apply(float* x, const uint32_t* counts, size_t M, size_t d,
                            size_t ldc, float delta, void* stream);
 
+/* "Majority vote with abstention" (Discussion section): ternary {-1, 0, +1}
+ * messages in both directions.  The paper describes the scheme in words and gives
+ * no thresholds; the two below (tau, quorum) are this library's definition.
+ * A ternary vector travels as two bit planes with the layout of a sign row:
+ * `sign` (bit = !(v < 0)) and `active` (bit set = a vote was cast).
+ *
+ * Worker side: v = g (m == NULL, beta == 0) or the updated momentum (as in
+ * ssgd_signum_momentum_pack, m updated in place); the worker abstains on element
+ * i when |v_i| < tau.  tau >= 0, finite; tau == 0 never abstains, and the sign
+ * plane always equals the 1-bit words of ssgd_sign_pack / ssgd_signum_momentum_pack.
+ *   sign_bits, active_bits out [M][ldw].                                       */
+ssgd_status ssgd_ternary_pack(const float* g, float* m, size_t M, size_t d, size_t ld,
+                              float beta, float tau, uint32_t* sign_bits,
+                              uint32_t* active_bits, size_t ldw, void* stream);
+
+/* Server side: with P / N the numbers of active +1 / -1 votes on a parameter, the
+ * answer is sign(P - N) when |P - N| >= max(quorum, 1) ("quorum reached") and 0
+ * otherwise (too many workers disagreed or abstained; a tie never decides).
+ *   vote_active out [W]: bit set = a decision was taken;
+ *   vote_sign   out [W]: bit set = decided +1 (0 where undecided).             */
+ssgd_status ssgd_quorum_vote(const uint32_t* sign_bits, const uint32_t* active_bits,
+                             size_t M, size_t d, size_t ldw, size_t quorum,
+                             uint32_t* vote_sign, uint32_t* vote_active, void* stream);
+
+/* Worker side: x[i] <- x[i] -/+ delta where vote_active is set (by vote_sign as
+ * in ssgd_sign_apply); x[i] unchanged where the server answered 0.             */
+ssgd_status ssgd_ternary_apply(float* x, const uint32_t* vote_sign,
+                               const uint32_t* vote_active, size_t d, float delta,
+                               void* stream);
+
+/* Section 3, "density" of a vector: phi(v) = |v|_1^2 / (d |v|_2^2), 1 for a fully
+ * dense vector and 1/d for a one-hot one.  ssgd_density_sums leaves
+ *   sums[0] = sum_i |t_i|,  sums[1] = sum_i t_i^2      (DEVICE double[2], 16-byte
+ * aligned, overwritten) with t = v when root == 0 and t = sqrt(v) when root != 0
+ * (v >= 0 then; used for the noise vector, see below), accumulated in fp64; the
+ * order of the additions is not fixed, so the last bits may vary from call to
+ * call.  phi = ssgd_density_from_sums(sums[0], sums[1], d) on the host (0 when
+ * d == 0 or the vector is all zero).                                           */
+ssgd_status ssgd_density_sums(const float* v, size_t d, int root, double* sums, void* stream);
+double ssgd_density_from_sums(double l1, double l2_squared, size_t d);
+
+/* Section 3: Welford's single-pass algorithm for the mean gradient g and its
+ * per-component variance.  Folds the n-th sample (n counts from 1, n <= 2^24)
+ * into the running state, in place, per element, in fp32:
+ *   d1 = g - mean;  mean <- mean + d1 / n;  d2 = g - mean;  m2 <- fma(d1, d2, m2).
+ * After n samples mean is the sample mean and m2 / (n - 1) the sample variance;
+ * the noise density phi(sigma) is ssgd_density_sums(m2, d, root = 1) since the
+ * factor 1 / (n - 1) cancels in phi.  Start from mean = m2 = 0.
+ *   g in [d];  mean, m2 in/out [d].                                            */
+ssgd_status ssgd_welford_update(const float* g, size_t n, float* mean, float* m2,
+                                size_t d, void* stream);
+
 /* ssgd_signsgd_step for a caller whose gradients live in HOST memory
  * (Algorithm 3's "independent gradient estimate" arriving from outside the
  * device): copies g_host to the device staging buffer, runs the step, and

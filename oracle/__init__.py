@@ -47,6 +47,8 @@ def _load():
     sz, f32, vp = ctypes.c_size_t, ctypes.c_float, ctypes.c_void_p
     L.ssgd_words_ref.restype = sz
     L.ssgd_words_ref.argtypes = [sz]
+    L.ssgd_density_ref.restype = ctypes.c_double
+    L.ssgd_density_ref.argtypes = [vp, sz, vp, vp]
     L.ssgd_count_planes_ref.restype = sz
     L.ssgd_count_planes_ref.argtypes = [sz]
     L.ssgd_warmup_steps_ref.restype = sz
@@ -60,6 +62,10 @@ def _load():
         "ssgd_signum_momentum_pack_ref": [vp, vp, sz, sz, sz, f32, vp, sz],
         "ssgd_signum_warmup_pack_ref": [vp, vp, sz, sz, sz, f32, vp, sz],
         "ssgd_signsgd_warmup_step_ref": [vp, vp, vp, sz, sz, sz, f32, f32, vp, sz, vp],
+        "ssgd_ternary_pack_ref": [vp, vp, sz, sz, sz, f32, f32, vp, vp, sz],
+        "ssgd_quorum_vote_ref": [vp, vp, sz, sz, sz, sz, vp, vp],
+        "ssgd_ternary_apply_ref": [vp, vp, vp, sz, f32],
+        "ssgd_welford_update_ref": [vp, sz, vp, vp, sz],
         "ssgd_vote_counts_ref": [vp, sz, sz, sz, vp],
         "ssgd_vote_count_planes_ref": [vp, sz, sz, sz, vp, sz],
         "ssgd_sum_apply_ref": [vp, vp, sz, sz, sz, f32],
@@ -242,3 +248,51 @@ def sum_apply(x: np.ndarray, counts: np.ndarray, M: int, d: int, delta: float,
     _load().ssgd_sum_apply_ref(_chk(x, np.float32, d, "x", True),
                                _chk(counts, np.uint32, count_planes(M) * ldc, "counts"),
                                M, d, ldc, delta)
+
+
+def ternary_pack(g: np.ndarray, m: np.ndarray | None, M: int, d: int, beta: float, tau: float,
+                 ld: int | None = None, ldw: int | None = None):
+    """Abstaining worker (Discussion; thresholds are this code base's): returns (sign, active) planes.
+    Parity with the paper unpinned: the paper gives no threshold."""
+    ld, ldw = _rows(M, d, ld, ldw)
+    sb = np.zeros(M * ldw, dtype=np.uint32)
+    ab = np.zeros(M * ldw, dtype=np.uint32)
+    mp = None if m is None else _chk(m, np.float32, M * ld, "m", True)
+    _load().ssgd_ternary_pack_ref(_chk(g, np.float32, M * ld, "g"), mp, M, d, ld, beta, tau,
+                                  sb.ctypes.data, ab.ctypes.data, ldw)
+    return sb, ab
+
+
+def quorum_vote(sign_bits: np.ndarray, active_bits: np.ndarray, M: int, d: int, quorum: int,
+                ldw: int | None = None):
+    """Server with quorum: returns (vote_sign, vote_active).  Parity with the paper unpinned."""
+    _, ldw = _rows(M, d, None, ldw)
+    vs = np.empty(words(d), dtype=np.uint32)
+    va = np.empty(words(d), dtype=np.uint32)
+    _load().ssgd_quorum_vote_ref(_chk(sign_bits, np.uint32, M * ldw, "sign_bits"),
+                                 _chk(active_bits, np.uint32, M * ldw, "active_bits"), M, d, ldw, quorum,
+                                 vs.ctypes.data, va.ctypes.data)
+    return vs, va
+
+
+def ternary_apply(x: np.ndarray, vote_sign: np.ndarray, vote_active: np.ndarray, d: int,
+                  delta: float) -> None:
+    """x moves by -/+ delta where the server decided, stays elsewhere.  Parity with the paper unpinned."""
+    _load().ssgd_ternary_apply_ref(_chk(x, np.float32, d, "x", True),
+                                   _chk(vote_sign, np.uint32, words(d), "vote_sign"),
+                                   _chk(vote_active, np.uint32, words(d), "vote_active"), d, delta)
+
+
+def density(v: np.ndarray):
+    """phi(v) = |v|_1^2 / (d |v|_2^2) of Sec. 3; returns (phi, |v|_1, |v|_2^2)."""
+    l1, l2 = ctypes.c_double(), ctypes.c_double()
+    phi = _load().ssgd_density_ref(_chk(v, np.float32, v.size, "v"), v.size, ctypes.addressof(l1),
+                                   ctypes.addressof(l2))
+    return float(phi), l1.value, l2.value
+
+
+def welford_update(g: np.ndarray, n: int, mean: np.ndarray, m2: np.ndarray) -> None:
+    """Welford's update with the n-th sample (n from 1), in place on mean and m2 (Sec. 3)."""
+    d = g.size
+    _load().ssgd_welford_update_ref(_chk(g, np.float32, d, "g"), n, _chk(mean, np.float32, d, "mean", True),
+                                    _chk(m2, np.float32, d, "m2", True), d)

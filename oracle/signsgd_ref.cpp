@@ -27,7 +27,11 @@
 //
 // All pointers are HOST pointers.  Parity status: every function below is
 // pinned by tests that do not call back into this file (brute force in Python,
-// closed forms in extended precision, invariants, bitwise MAJ3).
+// closed forms in extended precision, invariants, bitwise MAJ3) -- except that
+// the three abstention functions (ssgd_ternary_pack_ref, ssgd_quorum_vote_ref,
+// ssgd_ternary_apply_ref) are "parity unpinned" against the paper, which gives
+// their scheme in words without thresholds; they are pinned to the definition
+// stated above them.
 
 #include <cmath>
 #include <cstddef>
@@ -204,6 +208,96 @@ void ssgd_sum_apply_ref(float* x, const uint32_t* counts, size_t M, size_t d,
   for (size_t i = 0; i < d; ++i) {
     const float sum_of_signs = float(2 * P[i] - int32_t(M));
     x[i] = std::fmaf(-delta, sum_of_signs, x[i]);   // x - delta * sum, rounded once
+  }
+}
+
+// ---- majority vote with abstention (Discussion section) ------------------------
+// The paper states the scheme in words: a worker sends its vote "unless [it is]
+// very unsure about the sign of the true gradient in which case [it] send[s]
+// zero"; the server "counts the votes, and if quorum is not reached (i.e. too many
+// workers disagreed or abstained) [it] sends back zero".  No thresholds are given,
+// so the two used here are a definition of this code base, not the paper's:
+// a worker is unsure when |v| < tau; quorum is reached when |P - N| >= max(Q, 1),
+// P / N being the numbers of +1 / -1 votes cast.  (Parity with the paper is
+// therefore unpinned for these three functions; they are pinned to this
+// definition by brute force.)
+
+void ssgd_ternary_pack_ref(const float* g, float* m, size_t M, size_t d, size_t ld,
+                           float beta, float tau, uint32_t* sign_bits,
+                           uint32_t* active_bits, size_t ldw) {
+  std::vector<uint8_t> s(d), a(d);
+  for (size_t w = 0; w < M; ++w) {
+    const float* v = g + w * ld;
+    if (m != nullptr) {
+      ssgd_momentum_ref(g + w * ld, m + w * ld, d, beta);
+      v = m + w * ld;
+    }
+    ssgd_sign_unpacked_ref(v, d, s.data());
+    for (size_t i = 0; i < d; ++i) a[i] = (std::fabs(v[i]) < tau) ? 0 : 1;
+    ssgd_pack_bits_ref(s.data(), d, sign_bits + w * ldw);
+    ssgd_pack_bits_ref(a.data(), d, active_bits + w * ldw);
+  }
+}
+
+void ssgd_quorum_vote_ref(const uint32_t* sign_bits, const uint32_t* active_bits,
+                          size_t M, size_t d, size_t ldw, size_t quorum,
+                          uint32_t* vote_sign, uint32_t* vote_active) {
+  std::vector<uint8_t> s(d), a(d), vs(d), va(d);
+  std::vector<int32_t> diff(d, 0);   // P - N
+  for (size_t w = 0; w < M; ++w) {
+    ssgd_unpack_bits_ref(sign_bits + w * ldw, d, s.data());
+    ssgd_unpack_bits_ref(active_bits + w * ldw, d, a.data());
+    for (size_t i = 0; i < d; ++i) {
+      if (a[i]) diff[i] += s[i] ? 1 : -1;
+    }
+  }
+  const long long Q = quorum < 1 ? 1 : (long long)quorum;
+  for (size_t i = 0; i < d; ++i) {
+    const long long margin = diff[i] < 0 ? -(long long)diff[i] : (long long)diff[i];
+    va[i] = margin >= Q ? 1 : 0;
+    vs[i] = (va[i] && diff[i] > 0) ? 1 : 0;
+  }
+  ssgd_pack_bits_ref(vs.data(), d, vote_sign);
+  ssgd_pack_bits_ref(va.data(), d, vote_active);
+}
+
+void ssgd_ternary_apply_ref(float* x, const uint32_t* vote_sign,
+                            const uint32_t* vote_active, size_t d, float delta) {
+  std::vector<uint8_t> s(d), a(d);
+  ssgd_unpack_bits_ref(vote_sign, d, s.data());
+  ssgd_unpack_bits_ref(vote_active, d, a.data());
+  for (size_t i = 0; i < d; ++i) {
+    if (!a[i]) continue;           // the server answered 0: no move
+    if (s[i]) x[i] = x[i] - delta;
+    else      x[i] = x[i] + delta;
+  }
+}
+
+// ---- Section 3: density of a vector and Welford's mean / variance ---------------
+
+// phi(v) = |v|_1^2 / (d |v|_2^2); the two norms are returned too (fp64 sums).
+double ssgd_density_ref(const float* v, size_t d, double* l1_out, double* l2sq_out) {
+  double l1 = 0.0, l2sq = 0.0;
+  for (size_t i = 0; i < d; ++i) {
+    l1 += std::fabs((double)v[i]);
+    l2sq += (double)v[i] * (double)v[i];
+  }
+  if (l1_out) *l1_out = l1;
+  if (l2sq_out) *l2sq_out = l2sq;
+  if (d == 0 || !(l2sq > 0.0)) return 0.0;
+  return l1 * l1 / ((double)d * l2sq);
+}
+
+// Welford's update with the n-th sample (n counts from 1), per element, in fp32:
+// the textbook recurrence  mean_n = mean_{n-1} + (g - mean_{n-1}) / n,
+// M2_n = M2_{n-1} + (g - mean_{n-1}) (g - mean_n), the last line as one fma.
+void ssgd_welford_update_ref(const float* g, size_t n, float* mean, float* m2, size_t d) {
+  const float nf = (float)n;
+  for (size_t i = 0; i < d; ++i) {
+    const float d1 = g[i] - mean[i];
+    mean[i] = mean[i] + d1 / nf;
+    const float d2 = g[i] - mean[i];
+    m2[i] = std::fmaf(d1, d2, m2[i]);
   }
 }
 

@@ -42,6 +42,8 @@ def lib() -> ctypes.CDLL:
     sz, f32, vp, ci = ctypes.c_size_t, ctypes.c_float, ctypes.c_void_p, ctypes.c_int
     L.ssgd_words.restype = sz
     L.ssgd_words.argtypes = [sz]
+    L.ssgd_density_from_sums.restype = ctypes.c_double
+    L.ssgd_density_from_sums.argtypes = [ctypes.c_double, ctypes.c_double, sz]
     L.ssgd_count_planes.restype = sz
     L.ssgd_count_planes.argtypes = [sz]
     L.ssgd_warmup_steps.restype = sz
@@ -58,6 +60,11 @@ def lib() -> ctypes.CDLL:
         "ssgd_signsgd_warmup_step": [vp, vp, vp, sz, sz, sz, f32, f32, vp, sz, vp, vp],
         "ssgd_vote_counts": [vp, sz, sz, sz, vp, sz, vp],
         "ssgd_sum_apply": [vp, vp, sz, sz, sz, f32, vp],
+        "ssgd_ternary_pack": [vp, vp, sz, sz, sz, f32, f32, vp, vp, sz, vp],
+        "ssgd_quorum_vote": [vp, vp, sz, sz, sz, sz, vp, vp, vp],
+        "ssgd_ternary_apply": [vp, vp, vp, sz, f32, vp],
+        "ssgd_welford_update": [vp, sz, vp, vp, sz, vp],
+        "ssgd_density_sums": [vp, sz, ci, vp, vp],
         "ssgd_signsgd_step_host": [vp, vp, vp, sz, sz, sz, f32, f32, vp, vp, sz, vp, vp, vp],
         "ssgd_signsgd_step_noalloc": [vp, vp, vp, sz, sz, sz, f32, f32, vp],
     }
@@ -205,6 +212,60 @@ def sum_apply(x: torch.Tensor, counts: torch.Tensor, M: int, d: int, ldc: int, d
     _need(x, d, "x"); _need(counts, count_planes(M) * ldc, "counts")
     _check(lib().ssgd_sum_apply(_ptr(x, torch.float32, "x"), _ptr(counts, WORD_DTYPE, "counts"), M, d,
                                 ldc, delta, _stream(stream)), "ssgd_sum_apply")
+
+
+def ternary_pack(g: torch.Tensor, m: Optional[torch.Tensor], M: int, d: int, ld: int, beta: float,
+                 tau: float, sign_bits: torch.Tensor, active_bits: torch.Tensor, ldw: int,
+                 stream=None) -> None:
+    """Abstaining worker (Discussion): sign plane as in the 1-bit path, active plane = !(|v| < tau)."""
+    _need(g, M * ld, "g"); _need(sign_bits, M * ldw, "sign_bits"); _need(active_bits, M * ldw, "active_bits")
+    if m is not None:
+        _need(m, M * ld, "m")
+    _check(lib().ssgd_ternary_pack(
+        _ptr(g, torch.float32, "g"), _ptr(m, torch.float32, "m"), M, d, ld, beta, tau,
+        _ptr(sign_bits, WORD_DTYPE, "sign_bits"), _ptr(active_bits, WORD_DTYPE, "active_bits"), ldw,
+        _stream(stream)), "ssgd_ternary_pack")
+
+
+def quorum_vote(sign_bits: torch.Tensor, active_bits: torch.Tensor, M: int, d: int, ldw: int, quorum: int,
+                vote_sign: torch.Tensor, vote_active: torch.Tensor, stream=None) -> None:
+    """Server with quorum: decided where |P - N| >= max(quorum, 1), sign of P - N there."""
+    _need(sign_bits, M * ldw, "sign_bits"); _need(active_bits, M * ldw, "active_bits")
+    _need(vote_sign, -(-d // 32), "vote_sign"); _need(vote_active, -(-d // 32), "vote_active")
+    _check(lib().ssgd_quorum_vote(
+        _ptr(sign_bits, WORD_DTYPE, "sign_bits"), _ptr(active_bits, WORD_DTYPE, "active_bits"), M, d, ldw,
+        quorum, _ptr(vote_sign, WORD_DTYPE, "vote_sign"), _ptr(vote_active, WORD_DTYPE, "vote_active"),
+        _stream(stream)), "ssgd_quorum_vote")
+
+
+def ternary_apply(x: torch.Tensor, vote_sign: torch.Tensor, vote_active: torch.Tensor, d: int, delta: float,
+                  stream=None) -> None:
+    """x moves by -/+ delta where the server decided, stays where it answered 0."""
+    _need(x, d, "x"); _need(vote_sign, -(-d // 32), "vote_sign"); _need(vote_active, -(-d // 32), "vote_active")
+    _check(lib().ssgd_ternary_apply(
+        _ptr(x, torch.float32, "x"), _ptr(vote_sign, WORD_DTYPE, "vote_sign"),
+        _ptr(vote_active, WORD_DTYPE, "vote_active"), d, delta, _stream(stream)), "ssgd_ternary_apply")
+
+
+def welford_update(g: torch.Tensor, n: int, mean: torch.Tensor, m2: torch.Tensor, d: int, stream=None) -> None:
+    """Fold the n-th gradient sample (n from 1) into the running mean and sum of squared deviations."""
+    _need(g, d, "g"); _need(mean, d, "mean"); _need(m2, d, "m2")
+    _check(lib().ssgd_welford_update(_ptr(g, torch.float32, "g"), n, _ptr(mean, torch.float32, "mean"),
+                                     _ptr(m2, torch.float32, "m2"), d, _stream(stream)), "ssgd_welford_update")
+
+
+def density(v: torch.Tensor, d: int, root: bool = False, sums: Optional[torch.Tensor] = None, stream=None) -> float:
+    """phi(v) = |v|_1^2 / (d |v|_2^2) (Sec. 3); with root=True the density of sqrt(v).
+
+    `sums` is a float64 device tensor of 2 elements used for the two norms (allocated here if not
+    given).  Waits for the result: this is a measurement call, not part of the step."""
+    _need(v, d, "v")
+    if sums is None:
+        sums = torch.zeros(2, dtype=torch.float64, device=v.device)
+    _check(lib().ssgd_density_sums(_ptr(v, torch.float32, "v"), d, 1 if root else 0,
+                                   _ptr(sums, torch.float64, "sums"), _stream(stream)), "ssgd_density_sums")
+    l1, l2 = sums.tolist()
+    return float(lib().ssgd_density_from_sums(l1, l2, d))
 
 
 def signsgd_step_host(x: torch.Tensor, g_host: torch.Tensor, m: Optional[torch.Tensor], M: int,

@@ -1,0 +1,268 @@
+// Device-side building blocks shared by the kernels of this library: 128-bit
+// accesses, the sign rule, the momentum arithmetic, the warp-level word assembly
+// and the bit-sliced vote counters.  Everything lives in an unnamed namespace, so
+// each translation unit that includes this file gets its own copy.
+#ifndef SSGD_DEVICE_COMMON_CUH_
+#define SSGD_DEVICE_COMMON_CUH_
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace {
+
+// ---------------------------------------------------------------------------
+// small device helpers
+
+// 128-bit accesses.  Loads use the default caching path and stores the streaming
+// one: measured on B200 this pair, with one tile per CTA, streams faster than a
+// device-to-device copy, while evict-first loads and persistent grids were 8-10 %
+// slower.
+__device__ __forceinline__ float4 ld128(const float* p) {
+  return *reinterpret_cast<const float4*>(p);
+}
+__device__ __forceinline__ void st128(float* p, float4 v) {
+  __stcs(reinterpret_cast<float4*>(p), v);
+}
+
+// sign(.) of Algorithms 1-3 in one bit: +0, -0 and NaN all count as +1.
+__device__ __forceinline__ unsigned sign_bit(float v) { return (v < 0.0f) ? 0u : 1u; }
+
+__device__ __forceinline__ unsigned sign_nibble(const float4& v) {
+  return sign_bit(v.x) | (sign_bit(v.y) << 1) | (sign_bit(v.z) << 2) | (sign_bit(v.w) << 3);
+}
+
+// Algorithm 2, second step, as two correctly rounded fp32 operations.  Written
+// with explicit intrinsics so that the compiler can neither contract nor split them.
+__device__ __forceinline__ float momentum_update(float beta, float omb, float m, float g) {
+  return __fmaf_rn(beta, m, __fmul_rn(omb, g));
+}
+__device__ __forceinline__ float4 momentum_update4(float beta, float omb, const float4& m, const float4& g) {
+  return make_float4(momentum_update(beta, omb, m.x, g.x), momentum_update(beta, omb, m.y, g.y),
+                     momentum_update(beta, omb, m.z, g.z), momentum_update(beta, omb, m.w, g.w));
+}
+
+// Algorithm 3, worker block: four parameters move by -delta or +delta according
+// to four voted bits (bit set = sign +1 = subtract delta).
+__device__ __forceinline__ float4 apply4(const float4& x, unsigned nib, float delta, float minus) {
+  return make_float4(__fadd_rn(x.x, (nib & 1u) ? minus : delta), __fadd_rn(x.y, (nib & 2u) ? minus : delta),
+                     __fadd_rn(x.z, (nib & 4u) ? minus : delta), __fadd_rn(x.w, (nib & 8u) ? minus : delta));
+}
+
+// A warp holds 128 consecutive elements, lane l the four elements 4l..4l+3.
+// Lane l's four sign bits are bits 4(l%8)..4(l%8)+3 of word l/8, so an OR over
+// each group of eight lanes assembles the four canonical words; every lane of a
+// group receives its group's word.
+__device__ __forceinline__ unsigned assemble_word(unsigned nibble, unsigned lane) {
+  const unsigned group_mask = 0xFFu << (lane & 24u);
+  return __reduce_or_sync(group_mask, nibble << (4u * (lane & 7u)));
+}
+
+// Tiling shared by the worker, apply and fused kernels: a CTA of kThreads threads
+// owns a tile of kThreads * 4 * UNROLL consecutive elements of one row, a warp
+// 128 * UNROLL consecutive elements of it ("span"), so that a warp's words are
+// consecutive too: its span covers words (e0 / 32) + 4u + j for unroll step u and
+// lane group j = lane / 8.
+constexpr int kThreads = 256;
+
+// What a worker sends, and whether it keeps a momentum:
+//   kSignSGD       bit = sign(g)                       (Algorithm 1 / Algorithm 3 as printed)
+//   kSignum        m <- beta m + (1-beta) g, bit = sign(m)            (Algorithm 2)
+//   kSignumWarmup  m updated as in kSignum, bit = sign(g): the first C(beta)
+//                  iterations of Theorem 3, which accumulate the momentum as
+//                  normal but step with the sign of the stochastic gradient
+constexpr int kSignSGD = 0;
+constexpr int kSignum = 1;
+constexpr int kSignumWarmup = 2;
+
+// Within a group of eight lanes all lanes hold the same assembled word.  Lane
+// (lane % 8) == u keeps the word of unroll step u ("its" word), so that after the
+// UNROLL steps the 4 * UNROLL words of the span sit in 4 * UNROLL distinct lanes
+// and can be stored, or counted, once each.
+template <int UNROLL>
+__device__ __forceinline__ unsigned long long own_word_index(unsigned lane) {
+  return (unsigned long long)(lane & 7u) * 4u + (lane >> 3);   // valid for lane % 8 < UNROLL
+}
+
+// ---------------------------------------------------------------------------
+// majority vote: bit-sliced vertical counter
+//
+// The count of set bits per parameter is kept as NP bit-planes (plane p holds
+// bit p of 32 counters per word), and rows are folded in with carry-save adders
+// (3 words in, sum + carry out: one XOR3 and one MAJ3 per word), eight rows per
+// block, so the cost is about two logic operations per input word.
+//
+// The comparison with the threshold T = ceil(M/2) is folded into the counter's
+// start value: with L = NP - 1 chosen so that floor(M/2) < 2^L, the counter
+// starts at 2^L - T and can reach at most 2^L - T + M < 2^(L+1); its top plane
+// is then exactly [P >= T], the voted bit (ties, 2P = M, included).
+
+struct W4 {
+  unsigned x, y, z, w;
+};
+__device__ __forceinline__ W4 ld_words(const uint32_t* p) {
+  const uint4 v = *reinterpret_cast<const uint4*>(p);
+  return W4{v.x, v.y, v.z, v.w};
+}
+__device__ __forceinline__ unsigned xor3(unsigned a, unsigned b, unsigned c) { return a ^ b ^ c; }
+__device__ __forceinline__ unsigned maj3(unsigned a, unsigned b, unsigned c) {
+  return (a & b) | (c & (a | b));
+}
+// carry-save adder on 4 words: lo <- a ^ b ^ lo, returns the carries
+__device__ __forceinline__ W4 csa(W4& lo, const W4& a, const W4& b) {
+  W4 hi{maj3(lo.x, a.x, b.x), maj3(lo.y, a.y, b.y), maj3(lo.z, a.z, b.z), maj3(lo.w, a.w, b.w)};
+  lo = W4{xor3(lo.x, a.x, b.x), xor3(lo.y, a.y, b.y), xor3(lo.z, a.z, b.z), xor3(lo.w, a.w, b.w)};
+  return hi;
+}
+
+template <int NP>
+struct Counter {
+  W4 c[NP];
+  // add a word of weight 2^K: ripple from plane K upwards
+  template <int K>
+  __device__ __forceinline__ void add(W4 v) {
+#pragma unroll
+    for (int p = K; p < NP; ++p) {
+      const W4 carry{c[p].x & v.x, c[p].y & v.y, c[p].z & v.z, c[p].w & v.w};
+      c[p] = W4{c[p].x ^ v.x, c[p].y ^ v.y, c[p].z ^ v.z, c[p].w ^ v.w};
+      v = carry;
+    }
+  }
+  __device__ __forceinline__ void add2(const W4& a, const W4& b) {
+    if (NP >= 2) {
+      const W4 h = csa(c[0], a, b);
+      add<1>(h);
+    }
+  }
+  __device__ __forceinline__ void add4(const W4* a) {
+    if (NP >= 3) {
+      const W4 hA = csa(c[0], a[0], a[1]);
+      const W4 hB = csa(c[0], a[2], a[3]);
+      const W4 q = csa(c[1], hA, hB);
+      add<2>(q);
+    }
+  }
+  __device__ __forceinline__ void add8(const W4* a) {
+    if (NP >= 4) {
+      const W4 hA = csa(c[0], a[0], a[1]);
+      const W4 hB = csa(c[0], a[2], a[3]);
+      const W4 qA = csa(c[1], hA, hB);
+      const W4 hC = csa(c[0], a[4], a[5]);
+      const W4 hD = csa(c[0], a[6], a[7]);
+      const W4 qB = csa(c[1], hC, hD);
+      const W4 e = csa(c[2], qA, qB);
+      add<3>(e);
+    }
+  }
+};
+
+// The same counter on a single word per thread (used by the fused step kernel).
+template <int NP>
+struct Counter1 {
+  unsigned c[NP];
+  __device__ __forceinline__ void init(unsigned start_value) {
+#pragma unroll
+    for (int p = 0; p < NP; ++p) c[p] = ((start_value >> p) & 1u) ? 0xFFFFFFFFu : 0u;
+  }
+  template <int K>
+  __device__ __forceinline__ void add(unsigned v) {
+#pragma unroll
+    for (int p = K; p < NP; ++p) {
+      const unsigned carry = c[p] & v;
+      c[p] ^= v;
+      v = carry;
+    }
+  }
+  __device__ __forceinline__ void add2(unsigned a, unsigned b) {
+    if (NP >= 2) {
+      const unsigned h = maj3(c[0], a, b);
+      c[0] = xor3(c[0], a, b);
+      add<1>(h);
+    } else {
+      add<0>(a);   // not reached: one plane means one row
+    }
+  }
+  __device__ __forceinline__ unsigned top() const { return c[NP - 1]; }
+};
+
+// Four words of one output plane; bits at positions >= d are written as 0,
+// whatever the rows held there, and words at or beyond ceil(d/32) are not written.
+__device__ __forceinline__ void store_plane_words(uint32_t* __restrict__ out, unsigned long long q,
+                                                  unsigned long long d, const W4& v) {
+  const unsigned long long first = q * 128;  // first parameter of this chunk
+  if (first + 128 <= d) {
+    *reinterpret_cast<uint4*>(out + 4 * q) = make_uint4(v.x, v.y, v.z, v.w);
+  } else {
+    const unsigned w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const unsigned long long lo = first + 32ull * k;
+      if (lo < d) {
+        const unsigned long long left = d - lo;
+        const unsigned mask = left >= 32 ? 0xFFFFFFFFu : ((1u << left) - 1u);
+        out[4 * q + k] = w[k] & mask;
+      }
+    }
+  }
+}
+
+// One thread owns four consecutive words (one 128-bit load per row) and walks
+// down the M rows; one 256-thread CTA covers 1024 words.
+//   COUNTS = false: out[W] receives the top plane, the voted bit (Algorithm 3).
+//   COUNTS = true:  the counter starts at 0 and all NP planes are written,
+//                   plane p at out + p * ldc: the number of +1 votes per parameter,
+//                   bit-sliced, which is what the server sends back in the "(good)"
+//                   scheme of Section 4.
+template <int NP, bool COUNTS>
+__global__ void __launch_bounds__(kThreads)
+vote_kernel(const uint32_t* __restrict__ bits, unsigned M, unsigned long long d,
+            unsigned long long W, unsigned long long ldw, uint32_t* __restrict__ out,
+            unsigned long long ldc, unsigned start_value) {
+  const unsigned long long chunks = (W + 3) / 4;
+  const unsigned long long stride = (unsigned long long)gridDim.x * kThreads;
+  for (unsigned long long q = (unsigned long long)blockIdx.x * kThreads + threadIdx.x;
+       q < chunks; q += stride) {
+    const uint32_t* col = bits + 4 * q;
+    Counter<NP> cnt;
+#pragma unroll
+    for (int p = 0; p < NP; ++p) {
+      const unsigned f = ((start_value >> p) & 1u) ? 0xFFFFFFFFu : 0u;
+      cnt.c[p] = W4{f, f, f, f};
+    }
+    unsigned w = 0;
+    if (NP >= 4) {
+      for (; w + 8 <= M; w += 8) {
+        W4 a[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) a[k] = ld_words(col + (unsigned long long)(w + k) * ldw);
+        cnt.add8(a);
+      }
+    }
+    if (NP >= 3 && w + 4 <= M) {
+      W4 a[4];
+#pragma unroll
+      for (int k = 0; k < 4; ++k) a[k] = ld_words(col + (unsigned long long)(w + k) * ldw);
+      cnt.add4(a);
+      w += 4;
+    }
+    if (NP >= 2 && w + 2 <= M) {
+      const W4 a = ld_words(col + (unsigned long long)w * ldw);
+      const W4 b = ld_words(col + (unsigned long long)(w + 1) * ldw);
+      cnt.add2(a, b);
+      w += 2;
+    }
+    if (w < M) {
+      cnt.template add<0>(ld_words(col + (unsigned long long)w * ldw));
+      w += 1;
+    }
+    if (COUNTS) {
+#pragma unroll
+      for (int p = 0; p < NP; ++p) store_plane_words(out + (unsigned long long)p * ldc, q, d, cnt.c[p]);
+    } else {
+      store_plane_words(out, q, d, cnt.c[NP - 1]);
+    }
+  }
+}
+
+}  // namespace
+
+#endif  // SSGD_DEVICE_COMMON_CUH_

@@ -135,6 +135,37 @@ def test_good_scheme_argument_checks(L):
     assert a(A, A, 3, 0, 0, 0.1, None) == OK
 
 
+def test_abstention_argument_checks(L):
+    t = L.ssgd_ternary_pack
+    assert t(None, A, 1, 64, 64, 0.9, 0.1, A, A, 4, None) == NULL
+    assert t(A, None, 1, 64, 64, 0.9, 0.1, A, A, 4, None) == NULL        # m required when beta > 0
+    assert t(A, None, 1, 0, 0, 0.0, 0.1, A, A, 0, None) == OK
+    assert t(A, A, 1, 64, 64, 0.9, -0.1, A, A, 4, None) == ARG           # tau < 0
+    assert t(A, A, 1, 64, 64, 0.9, float("nan"), A, A, 4, None) == ARG
+    assert t(A, A, 1, 64, 64, 0.9, 0.1, A + 4, A, 4, None) == ALIGN
+    q = L.ssgd_quorum_vote
+    assert q(A, None, 3, 64, 4, 1, A, A, None) == NULL
+    assert q(A, A, 0, 64, 4, 1, A, A, None) == SIZE
+    assert q(A, A, 3, 0, 0, 1, A, A, None) == OK
+    a = L.ssgd_ternary_apply
+    assert a(A, A, None, 64, 0.1, None) == NULL
+    assert a(A, A, A, 64, float("inf"), None) == ARG
+    assert a(A, A, A, 0, 0.1, None) == OK
+
+
+def test_statistics_argument_checks(L):
+    w = L.ssgd_welford_update
+    assert w(None, 1, A, A, 64, None) == NULL
+    assert w(A, 0, A, A, 64, None) == ARG                 # samples count from 1
+    assert w(A, (1 << 24) + 1, A, A, 64, None) == ARG
+    assert w(A + 4, 1, A, A, 64, None) == ALIGN
+    assert w(A, 1, A, A, 0, None) == OK
+    assert L.ssgd_density_sums(None, 64, 0, A, None) == NULL
+    assert L.ssgd_density_sums(A, 64, 0, A + 8, None) == ALIGN
+    f = L.ssgd_density_from_sums
+    assert f(4.0, 4.0, 4) == 1.0 and f(2.0, 4.0, 4) == 0.25 and f(0.0, 0.0, 4) == 0.0 and f(1.0, 1.0, 0) == 0.0
+
+
 def test_binding_refuses_to_run_without_the_library(monkeypatch, tmp_path):
     from paper_1802_04434_b200 import binding
     monkeypatch.setattr(binding, "_lib", None)

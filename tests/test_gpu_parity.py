@@ -431,3 +431,76 @@ def test_vote_counts_and_sum_apply(M):
         gx = f32(xd)
         assert_same_f32(gx[:d], x_ref, "x (M=%d d=%d)" % (M, d))
         assert np.all(gx[d:] == np.float32(CANARY_F))
+
+
+# ------------------------------------------------------------------ majority vote with abstention
+
+@pytest.mark.parametrize("M", [1, 2, 3, 7, 8, 16, 33, 255, 1024])
+def test_abstention_path(M):
+    for d in (1, 33, 1000, 4097, 70001 if M <= 33 else 3000):
+        ld, W = wl.round_up(d, 4), oracle.words(d)
+        ldw = wl.round_up(W, 4)
+        g, m, x = rand_inputs(M, d, ld, seed=M * 13 + d, special=True)
+        for beta, with_m, tau, Q in ((0.9, True, 0.05, 2), (0.0, False, 0.3, 0), (0.9, True, 0.0, 0), (0.0, False, 1.0, M // 2 + 1)):
+            gd, xd = torch.from_numpy(g).to(DEV), torch.from_numpy(x).to(DEV)
+            md = torch.from_numpy(m).to(DEV) if with_m else None
+            sb = torch.full((M, ldw), CANARY_WORD, dtype=torch.int32, device=DEV)
+            ab = torch.full((M, ldw), CANARY_WORD, dtype=torch.int32, device=DEV)
+            B.ternary_pack(gd, md, M, d, ld, beta, tau, sb, ab, ldw)
+            m_ref = m.copy().reshape(-1) if with_m else None
+            sb_ref, ab_ref = oracle.ternary_pack(g.reshape(-1), m_ref, M, d, beta, tau, ld=ld, ldw=ldw)
+            got_s, got_a = u32(sb), u32(ab)
+            assert np.array_equal(got_s[:, :W], sb_ref.reshape(M, ldw)[:, :W])
+            assert np.array_equal(got_a[:, :W], ab_ref.reshape(M, ldw)[:, :W])
+            assert np.all(got_s[:, W:] == np.uint32(0xDEADBEEF)) and np.all(got_a[:, W:] == np.uint32(0xDEADBEEF))
+            if with_m:
+                assert_same_f32(f32(md).reshape(-1), m_ref, "m")
+            sb[:, W:] = 0
+            ab[:, W:] = 0
+            vs = torch.full((W + 4,), CANARY_WORD, dtype=torch.int32, device=DEV)
+            va = torch.full((W + 4,), CANARY_WORD, dtype=torch.int32, device=DEV)
+            B.quorum_vote(sb, ab, M, d, ldw, Q, vs, va)
+            vs_ref, va_ref = oracle.quorum_vote(u32(sb).reshape(-1).copy(), u32(ab).reshape(-1).copy(), M, d, Q, ldw=ldw)
+            assert np.array_equal(u32(vs)[:W], vs_ref) and np.array_equal(u32(va)[:W], va_ref), (M, d, Q)
+            assert np.all(u32(vs)[W:] == np.uint32(0xDEADBEEF)) and np.all(u32(va)[W:] == np.uint32(0xDEADBEEF))
+            B.ternary_apply(xd, vs, va, d, 1e-3)
+            x_ref = x.copy()
+            oracle.ternary_apply(x_ref, vs_ref, va_ref, d, 1e-3)
+            assert_same_f32(f32(xd), x_ref, "x")
+
+
+# ------------------------------------------------------------------ Section 3: density and Welford
+
+@pytest.mark.parametrize("d", [1, 3, 1000, 4099, 1 << 20, (1 << 22) + 5])
+def test_welford_and_density(d):
+    r = np.random.default_rng(d)
+    n = 5
+    g = (0.3 + r.standard_normal((n, d))).astype(np.float32)
+    mean_d = torch.zeros(d, device=DEV)
+    m2_d = torch.zeros(d, device=DEV)
+    mean, m2 = np.zeros(d, dtype=np.float32), np.zeros(d, dtype=np.float32)
+    for k in range(n):
+        B.welford_update(torch.from_numpy(g[k]).to(DEV), k + 1, mean_d, m2_d, d)
+        oracle.welford_update(g[k], k + 1, mean, m2)
+    assert_same_f32(f32(mean_d), mean, "mean")
+    assert_same_f32(f32(m2_d), m2, "m2")
+    # the density is an fp64 sum of exactly representable terms in a different order than the
+    # oracle's: relative error is bounded by d * 2^-53, far inside 1e-11
+    phi_ref, l1, l2 = oracle.density(mean)
+    phi = B.density(mean_d, d)
+    assert abs(phi - phi_ref) <= 1e-11 * max(phi_ref, 1e-300)
+    sig = np.sqrt(m2.astype(np.float64)).astype(np.float32)      # sqrt in fp64, rounded once, as a stand-in
+    phi_s = B.density(m2_d, d, root=True)
+    l1s = float(np.sqrt(m2.astype(np.float64)).sum())
+    l2s = float(m2.astype(np.float64).sum())
+    assert abs(phi_s - l1s * l1s / (d * l2s)) <= 1e-11 * phi_s if l2s > 0 else phi_s == 0.0
+
+
+def test_density_of_dense_and_one_hot_vectors_gpu():
+    d = 1 << 20
+    dense = torch.full((d,), -0.75, device=DEV)
+    assert abs(B.density(dense, d) - 1.0) < 1e-12
+    one_hot = torch.zeros(d, device=DEV)
+    one_hot[12345] = 4.0
+    assert abs(B.density(one_hot, d) - 1.0 / d) < 1e-18
+    assert B.density(torch.zeros(8, device=DEV), 8) == 0.0

@@ -506,3 +506,138 @@ def test_sum_apply_is_x_minus_delta_times_sum_rounded_once():
     oracle.sum_apply(xa, one, 1, d, float(delta))
     oracle.sign_apply(xb, bits[:oracle.words(d)].copy(), d, float(delta))
     assert np.array_equal(xa, xb)
+
+
+# ---------------------------------------------------------------- vote with abstention
+# (the paper gives this scheme in words only; these tests pin the oracle to the stated definition:
+#  abstain when |v| < tau; decided when |P - N| >= max(Q, 1); sign of P - N)
+
+def test_abstention_rule_on_listed_values():
+    v = np.array([0.5, -0.5, 0.09, -0.09, 0.1, -0.1, 0.0, -0.0, np.nan, np.inf, -np.inf], dtype=np.float32)
+    sb, ab = oracle.ternary_pack(v, None, 1, v.size, 0.0, float(np.float32(0.1)))
+    assert oracle.unpack_bits(sb, v.size).tolist() == [1, 0, 1, 0, 1, 0, 1, 1, 1, 1, 0]
+    assert oracle.unpack_bits(ab, v.size).tolist() == [1, 1, 0, 0, 1, 1, 0, 0, 1, 1, 1]
+    sb0, ab0 = oracle.ternary_pack(v, None, 1, v.size, 0.0, 0.0)       # tau = 0 never abstains
+    assert np.array_equal(sb0, oracle.sign_pack(v, 1, v.size)) and oracle.unpack_bits(ab0, v.size).all()
+
+
+@pytest.mark.parametrize("M", [1, 2, 3, 4, 5, 6])
+def test_quorum_vote_all_ternary_patterns(M):
+    pats = list(itertools.product((-1, 0, 1), repeat=M))
+    d = len(pats)
+    sb = np.concatenate([np.array(py_pack([1 if p[w] > 0 else 0 for p in pats]), dtype=np.uint32) for w in range(M)])
+    ab = np.concatenate([np.array(py_pack([1 if p[w] != 0 else 0 for p in pats]), dtype=np.uint32) for w in range(M)])
+    for Q in (0, 1, 2, 3, M, M + 1, 50):
+        vs, va = oracle.quorum_vote(sb, ab, M, d, Q)
+        exp_a = [1 if abs(sum(p)) >= max(Q, 1) else 0 for p in pats]
+        exp_s = [1 if (abs(sum(p)) >= max(Q, 1) and sum(p) > 0) else 0 for p in pats]
+        assert va.tolist() == py_pack(exp_a) and vs.tolist() == py_pack(exp_s), (M, Q)
+
+
+def test_abstention_with_tau0_q0_equals_one_bit_path_away_from_ties():
+    r = rng(71)
+    M, d = 7, 3000
+    g = r.standard_normal((M, d)).astype(np.float32).reshape(-1)
+    m = (0.2 * r.standard_normal((M, d))).astype(np.float32).reshape(-1)
+    x = r.standard_normal(d).astype(np.float32)
+    m1, x1 = m.copy(), x.copy()
+    bits, vote = oracle.signsgd_step(x1, g, m1, M, d, 0.9, 1e-3)
+    m2, x2 = m.copy(), x.copy()
+    sb, ab = oracle.ternary_pack(g, m2, M, d, 0.9, 0.0)
+    vs, va = oracle.quorum_vote(sb, ab, M, d, 0)
+    oracle.ternary_apply(x2, vs, va, d, 1e-3)
+    assert np.array_equal(sb, bits) and np.array_equal(m1, m2)
+    assert oracle.unpack_bits(va, d).all()                     # odd M, nobody abstains: always decided
+    assert np.array_equal(vs, vote) and np.array_equal(x1, x2)
+
+
+def test_ternary_apply_moves_only_decided_elements():
+    r = rng(72)
+    d = 500
+    x = r.standard_normal(d).astype(np.float32)
+    s = r.integers(0, 2, d, dtype=np.uint8)
+    a = r.integers(0, 2, d, dtype=np.uint8)
+    got = x.copy()
+    oracle.ternary_apply(got, np.array(py_pack((s & a).tolist()), dtype=np.uint32),
+                         np.array(py_pack(a.tolist()), dtype=np.uint32), d, 0.25)
+    expect = [round_f32(Fraction(xi) + (0 if not ai else (Fraction(-1, 4) if si else Fraction(1, 4))))
+              for xi, si, ai in zip(x.tolist(), s.tolist(), a.tolist())]
+    assert got.tolist() == expect
+
+
+def test_abstention_shrinks_wrong_decisions_on_noisy_small_gradients():
+    # workers that abstain when unsure and a server that wants a margin decide less often, and when
+    # they do decide they are wrong less often than the plain majority: the point of the scheme
+    r = rng(73)
+    M, d = 15, 100_000
+    mu = np.float32(-0.2)
+    g = (mu + r.standard_normal((M, d))).astype(np.float32).reshape(-1)
+    plain = oracle.unpack_bits(oracle.majority_vote(oracle.sign_pack(g, M, d), M, d), d)
+    sb, ab = oracle.ternary_pack(g, None, M, d, 0.0, 0.5)
+    vs, va = oracle.quorum_vote(sb, ab, M, d, 3)
+    vs, va = oracle.unpack_bits(vs, d).astype(bool), oracle.unpack_bits(va, d).astype(bool)
+    assert 0.2 < va.mean() < 0.9
+    assert vs[va].mean() < plain.mean()          # true sign is negative: a set bit is a wrong decision
+
+
+# ---------------------------------------------------------------- Section 3: density and Welford
+
+def test_density_of_dense_and_one_hot_vectors():
+    # "for a fully dense vector phi = 1 and for a fully sparse vector phi = 1/d"
+    d = 1000
+    r = rng(81)
+    dense = (3.0 * r.choice([-1.0, 1.0], d)).astype(np.float32)
+    assert abs(oracle.density(dense)[0] - 1.0) < 1e-12
+    one_hot = np.zeros(d, dtype=np.float32)
+    one_hot[17] = -2.5
+    assert abs(oracle.density(one_hot)[0] - 1.0 / d) < 1e-15
+    assert oracle.density(np.zeros(5, dtype=np.float32))[0] == 0.0
+    # a Gaussian vector: E|z| = sqrt(2/pi), E z^2 = 1, so phi -> 2/pi
+    z = r.standard_normal(400_000).astype(np.float32)
+    phi, l1, l2 = oracle.density(z)
+    assert abs(phi - 2 / math.pi) < 5e-3
+    assert abs(l1 - float(np.abs(z.astype(np.float64)).sum())) < 1e-9 * l1
+    assert abs(l2 - float((z.astype(np.float64) ** 2).sum())) < 1e-9 * l2
+    # k equal non-zeros out of d: phi = k / d
+    v = np.zeros(d, dtype=np.float32)
+    v[:250] = 0.5
+    assert abs(oracle.density(v)[0] - 0.25) < 1e-12
+
+
+def test_welford_matches_two_pass_mean_and_variance():
+    r = rng(82)
+    n, d = 40, 3000
+    g = (1.5 + 2.0 * r.standard_normal((n, d))).astype(np.float32)
+    mean = np.zeros(d, dtype=np.float32)
+    m2 = np.zeros(d, dtype=np.float32)
+    for k in range(n):
+        oracle.welford_update(g[k], k + 1, mean, m2)
+    g64 = g.astype(np.float64)
+    assert np.allclose(mean, g64.mean(axis=0), rtol=0, atol=2e-6)
+    assert np.allclose(m2 / (n - 1), g64.var(axis=0, ddof=1), rtol=2e-5)
+    # the noise density needs no division: phi(sigma) = phi(sqrt(m2))
+    sigma = np.sqrt(m2 / np.float32(n - 1)).astype(np.float32)
+    assert abs(oracle.density(sigma)[0] - oracle.density(np.sqrt(m2).astype(np.float32))[0]) < 1e-6
+
+
+def test_welford_update_rounding_sequence():
+    r = rng(83)
+    d = 300
+    g = r.standard_normal(d).astype(np.float32)
+    mean = r.standard_normal(d).astype(np.float32)
+    m2 = np.abs(r.standard_normal(d)).astype(np.float32)
+    n = 7
+    expect_mean, expect_m2 = [], []
+    for gi, mu, s in zip(g.tolist(), mean.tolist(), m2.tolist()):
+        d1 = round_f32(Fraction(gi) - Fraction(mu))
+        q = round_f32(Fraction(d1) / n)
+        mu2 = round_f32(Fraction(mu) + Fraction(q))
+        d2 = round_f32(Fraction(gi) - Fraction(mu2))
+        expect_mean.append(mu2)
+        expect_m2.append(round_f32(Fraction(d1) * Fraction(d2) + Fraction(s)))
+    oracle.welford_update(g, n, mean, m2)
+    assert mean.tolist() == expect_mean and m2.tolist() == expect_m2
+    # first sample: mean becomes the sample, m2 stays 0
+    mean0, m20 = np.zeros(d, dtype=np.float32), np.zeros(d, dtype=np.float32)
+    oracle.welford_update(g, 1, mean0, m20)
+    assert np.array_equal(mean0, g) and not m20.any()
