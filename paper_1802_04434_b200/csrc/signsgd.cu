@@ -7,9 +7,16 @@
 //                   1/8 B of sign bits written); 4.125 B for the sign-only form
 //   vote kernel     (M + 1) / 8 B per parameter
 //   apply kernel    8.125 B per parameter
-// so the design rules are: 128-bit coalesced accesses, many independent loads
-// in flight per thread, streaming cache hints (nothing is re-read), grids sized
-// in whole waves of the SM count, and 64-bit indexing (M * d exceeds 2^32).
+//   fused step      12.125 M + 8.125 B per parameter (the three above in one
+//                   launch; the sign words are not read back)
+// No step is a contraction, so there is no tensor-core work.  The design rules
+// that measurement on B200 settled: 128-bit coalesced accesses, eight independent
+// loads in flight per thread, one tile per CTA (the hardware's CTA scheduler
+// balances DRAM channels better than a persistent grid-stride loop did), default
+// caching on loads and streaming stores, 64-bit indexing (M * d exceeds 2^32).
+// Staging tiles through shared memory with bulk asynchronous copies was tried for
+// the worker kernel and was 15-25 % slower than direct register loads: there is
+// no reuse for shared memory to serve, only an extra hop.
 
 #include "host_common.h"
 

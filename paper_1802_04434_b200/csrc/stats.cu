@@ -42,29 +42,39 @@ welford_kernel(const float* __restrict__ g, float* __restrict__ mean, float* __r
 // ROOT (then sums[1] is sum_i v_i): all that phi needs.  Accumulated in fp64:
 // per thread, then per warp by shuffles, per CTA through shared memory, and one
 // atomic add per CTA and quantity.
+constexpr int kDensityUnroll = 4;   // 128-bit loads in flight per thread
+
+template <bool ROOT>
+__device__ __forceinline__ void density_term(float t, double& l1, double& l2) {
+  const double td = (double)t;
+  if (ROOT) {
+    l1 += sqrt(td);
+    l2 += td;
+  } else {
+    l1 += fabs(td);
+    l2 = fma(td, td, l2);
+  }
+}
+
 template <bool ROOT>
 __global__ void __launch_bounds__(kThreads)
 density_sums_kernel(const float* __restrict__ v, unsigned long long d, double* __restrict__ sums) {
+  constexpr unsigned long long TILE = (unsigned long long)kThreads * 4 * kDensityUnroll;
   double l1 = 0.0, l2 = 0.0;
-  const unsigned long long stride = (unsigned long long)gridDim.x * kThreads * 4;
-  for (unsigned long long e = ((unsigned long long)blockIdx.x * kThreads + threadIdx.x) * 4; e < d; e += stride) {
-    float t[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-    if (e + 4 <= d) {
-      const float4 q = ld128(v + e);
-      t[0] = q.x; t[1] = q.y; t[2] = q.z; t[3] = q.w;
-    } else {
-      for (int k = 0; k < 4; ++k)
-        if (e + k < d) t[k] = v[e + k];
-    }
+  for (unsigned long long t0 = (unsigned long long)blockIdx.x * TILE; t0 < d; t0 += (unsigned long long)gridDim.x * TILE) {
+    if (t0 + TILE <= d) {
+      float4 q[kDensityUnroll];
 #pragma unroll
-    for (int k = 0; k < 4; ++k) {
-      if (ROOT) {
-        l1 += sqrt((double)t[k]);
-        l2 += (double)t[k];
-      } else {
-        l1 += fabs((double)t[k]);
-        l2 += (double)t[k] * (double)t[k];
+      for (int u = 0; u < kDensityUnroll; ++u) q[u] = ld128(v + t0 + (unsigned long long)u * kThreads * 4 + threadIdx.x * 4);
+#pragma unroll
+      for (int u = 0; u < kDensityUnroll; ++u) {
+        density_term<ROOT>(q[u].x, l1, l2);
+        density_term<ROOT>(q[u].y, l1, l2);
+        density_term<ROOT>(q[u].z, l1, l2);
+        density_term<ROOT>(q[u].w, l1, l2);
       }
+    } else {
+      for (unsigned long long i = t0 + threadIdx.x; i < d; i += kThreads) density_term<ROOT>(v[i], l1, l2);
     }
   }
 #pragma unroll
@@ -109,8 +119,8 @@ ssgd_status ssgd_density_sums(const float* v, size_t d, int root, double* sums, 
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (cudaMemsetAsync(sums, 0, 2 * sizeof(double), s) != cudaSuccess) return SSGD_ERR_CUDA;
   if (d == 0) return SSGD_OK;
-  // four float4 per thread and tile; the grid-stride loop covers the rest
-  unsigned long long ctas = ((d + 15) / 16 + kThreads - 1) / kThreads;
+  const unsigned long long tile = (unsigned long long)kThreads * 4 * kDensityUnroll;
+  const unsigned long long ctas = (d + tile - 1) / tile;
   if (root)
     density_sums_kernel<true><<<grid_for(ctas), kThreads, 0, s>>>(v, d, sums);
   else

@@ -88,6 +88,16 @@ ssgd_status launch_sum_apply(float* x, const uint32_t* counts, size_t M, size_t 
 //            vote_active and vote_sign (set only where active and positive);
 //   worker   moves x by -/+ delta where the answer is active, else leaves it.
 
+constexpr int kTernaryUnroll = 4;
+
+__device__ __forceinline__ unsigned active_nibble(const float4& v, float tau) {
+  return ((fabsf(v.x) < tau) ? 0u : 1u) | ((fabsf(v.y) < tau) ? 0u : 2u) | ((fabsf(v.z) < tau) ? 0u : 4u) |
+         ((fabsf(v.w) < tau) ? 0u : 8u);
+}
+
+// Same tiling as the worker kernel (one tile of kThreads * 16 elements of one row
+// per CTA, all loads of a thread issued before their first use), with a second
+// output plane.
 template <bool MOMENTUM>
 __global__ void __launch_bounds__(kThreads)
 ternary_pack_kernel(const float* __restrict__ g, float* __restrict__ m,
@@ -95,7 +105,7 @@ ternary_pack_kernel(const float* __restrict__ g, float* __restrict__ m,
                     unsigned long long d, unsigned long long ld, unsigned long long ldw,
                     unsigned long long tiles_per_row, unsigned long long total_tiles,
                     float beta, float omb, float tau) {
-  constexpr int UNROLL = 2;
+  constexpr int UNROLL = kTernaryUnroll;
   constexpr unsigned long long TILE = (unsigned long long)kThreads * 4 * UNROLL;
   constexpr unsigned SPAN = 128 * UNROLL;
   const unsigned lane = threadIdx.x & 31u;
@@ -109,46 +119,58 @@ ternary_pack_kernel(const float* __restrict__ g, float* __restrict__ m,
     float* mr = MOMENTUM ? m + row * ld : nullptr;
     uint32_t* sr = sign_bits + row * ldw + (e0 >> 5);
     uint32_t* ar = active_bits + row * ldw + (e0 >> 5);
-    const bool interior = e0 + SPAN <= d;
+    if (e0 + SPAN <= d) {
+      float4 gv[UNROLL], mv[UNROLL];
 #pragma unroll
-    for (int u = 0; u < UNROLL; ++u) {
-      const unsigned long long e = e0 + u * 128 + lane * 4;
-      float v[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-      bool have[4] = {interior, interior, interior, interior};
-      if (interior) {
-        float4 gv = ld128(gr + e);
+      for (int u = 0; u < UNROLL; ++u) gv[u] = ld128(gr + e0 + u * 128 + lane * 4);
+      if (MOMENTUM) {
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) mv[u] = ld128(mr + e0 + u * 128 + lane * 4);
+      }
+      unsigned smine = 0, amine = 0;
+#pragma unroll
+      for (int u = 0; u < UNROLL; ++u) {
+        float4 v = gv[u];
         if (MOMENTUM) {
-          gv = momentum_update4(beta, omb, ld128(mr + e), gv);
-          st128(mr + e, gv);
+          v = momentum_update4(beta, omb, mv[u], v);
+          st128(mr + e0 + u * 128 + lane * 4, v);
         }
-        v[0] = gv.x; v[1] = gv.y; v[2] = gv.z; v[3] = gv.w;
-      } else {
+        const unsigned sword = assemble_word(sign_nibble(v), lane);
+        const unsigned aword = assemble_word(active_nibble(v, tau), lane);
+        if ((lane & 7u) == (unsigned)u) {
+          smine = sword;
+          amine = aword;
+        }
+      }
+      if ((lane & 7u) < (unsigned)UNROLL) {
+        sr[own_word_index<UNROLL>(lane)] = smine;
+        ar[own_word_index<UNROLL>(lane)] = amine;
+      }
+    } else {
+      // ragged end of the row: element-wise guards; bits at positions >= d stay 0
+#pragma unroll 1
+      for (int u = 0; u < UNROLL; ++u) {
+        const unsigned long long e = e0 + u * 128 + lane * 4;
+        unsigned snib = 0, anib = 0;
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
-          have[k] = e + k < d;
-          if (have[k]) {
-            v[k] = gr[e + k];
+          if (e + k < d) {
+            float v = gr[e + k];
             if (MOMENTUM) {
-              v[k] = momentum_update(beta, omb, mr[e + k], v[k]);
-              mr[e + k] = v[k];
+              v = momentum_update(beta, omb, mr[e + k], v);
+              mr[e + k] = v;
             }
+            snib |= sign_bit(v) << k;
+            anib |= ((fabsf(v) < tau) ? 0u : 1u) << k;
           }
         }
-      }
-      unsigned snib = 0, anib = 0;
-#pragma unroll
-      for (int k = 0; k < 4; ++k) {
-        if (have[k]) {
-          snib |= sign_bit(v[k]) << k;
-          anib |= ((fabsf(v[k]) < tau) ? 0u : 1u) << k;
+        const unsigned sword = assemble_word(snib, lane);
+        const unsigned aword = assemble_word(anib, lane);
+        const unsigned long long first = e0 + u * 128 + (lane >> 3) * 32;  // first element of the word
+        if ((lane & 7u) == 0 && first < d) {
+          sr[u * 4 + (lane >> 3)] = sword;
+          ar[u * 4 + (lane >> 3)] = aword;
         }
-      }
-      const unsigned sword = assemble_word(snib, lane);
-      const unsigned aword = assemble_word(anib, lane);
-      const unsigned long long first = e0 + u * 128 + (lane >> 3) * 32;  // first element of the word
-      if ((lane & 7u) == 0 && first < d) {
-        sr[u * 4 + (lane >> 3)] = sword;
-        ar[u * 4 + (lane >> 3)] = aword;
       }
     }
   }
@@ -273,7 +295,7 @@ ssgd_status ssgd_ternary_pack(const float* g, float* m, size_t M, size_t d, size
   if (!beta_ok(beta) || !(tau >= 0.0f) || !isfinite(tau)) return SSGD_ERR_ARG;
   if (!m && beta != 0.0f) return SSGD_ERR_NULL;
   if (d == 0) return SSGD_OK;
-  constexpr unsigned long long TILE = (unsigned long long)kThreads * 4 * 2;
+  constexpr unsigned long long TILE = (unsigned long long)kThreads * 4 * kTernaryUnroll;
   const unsigned long long tiles_per_row = (d + TILE - 1) / TILE;
   const unsigned long long total = tiles_per_row * M;
   cudaStream_t s = static_cast<cudaStream_t>(stream);

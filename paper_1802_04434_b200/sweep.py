@@ -98,6 +98,47 @@ def run_point(d: int, M: int, reps: int, dev) -> list:
     return rows
 
 
+def run_variants(d: int, M: int, reps: int, dev) -> list:
+    """The calls beside the main path (warm-up, count planes, abstention, statistics) at one size."""
+    ld = (d + 3) // 4 * 4
+    W = (d + 31) // 32
+    ldw = (W + 3) // 4 * 4
+    NPc = B.count_planes(M)
+    g = torch.randn(M, ld, device=dev)
+    m = torch.zeros(M, ld, device=dev)
+    x = torch.randn(d, device=dev)
+    bits = torch.zeros(M, ldw, dtype=torch.int32, device=dev)
+    act = torch.zeros(M, ldw, dtype=torch.int32, device=dev)
+    counts = torch.zeros(NPc, ldw, dtype=torch.int32, device=dev)
+    vs = torch.zeros(W, dtype=torch.int32, device=dev)
+    va = torch.zeros(W, dtype=torch.int32, device=dev)
+    mean, m2 = torch.zeros(d, device=dev), torch.zeros(d, device=dev)
+    sums = torch.zeros(2, dtype=torch.float64, device=dev)
+    B.sign_pack(g, M, d, ld, bits, ldw)
+    rows = []
+
+    def rec(name, ms, nbytes):
+        gbs = nbytes / (ms * 1e-3) / 1e9
+        rows.append((d, M, name, ms * 1e3, gbs, gbs / peak_gbs(), int(nbytes >= 2 * L2_BYTES)))
+
+    rec("signum_warmup_pack", time_launches(lambda s: B.signum_warmup_pack(g, m, M, d, ld, 0.9, bits, ldw), 1, reps),
+        12.125 * M * d)
+    rec("vote_counts", time_launches(lambda s: B.vote_counts(bits, M, d, ldw, counts, ldw), 1, reps),
+        (M + NPc) / 8.0 * d)
+    rec("sum_apply", time_launches(lambda s: B.sum_apply(x, counts, M, d, ldw, 1e-4), 1, reps), (8 + NPc / 8.0) * d)
+    rec("ternary_pack", time_launches(lambda s: B.ternary_pack(g, m, M, d, ld, 0.9, 0.1, bits, act, ldw), 1, reps),
+        12.25 * M * d)
+    rec("quorum_vote", time_launches(lambda s: B.quorum_vote(bits, act, M, d, ldw, 2, vs, va), 1, reps),
+        (2 * M + 2) / 8.0 * d)
+    rec("ternary_apply", time_launches(lambda s: B.ternary_apply(x, vs, va, d, 1e-4), 1, reps), 8.25 * d)
+    rec("welford_update", time_launches(lambda s: B.welford_update(g[0], 3, mean, m2, d), 1, reps), 20.0 * d)
+    lib = B.lib()
+    sp, xp, st = sums.data_ptr(), x.data_ptr(), None
+    rec("density_sums", time_launches(lambda s: lib.ssgd_density_sums(xp, d, 0, sp, torch.cuda.current_stream().cuda_stream),
+                                      1, reps), 4.0 * d)
+    return rows
+
+
 def main(argv=None):
     ap = argparse.ArgumentParser()
     ap.add_argument("--min-log2", type=int, default=10)
@@ -105,6 +146,8 @@ def main(argv=None):
     ap.add_argument("--workers", default="1,3,7,15,31")
     ap.add_argument("--reps", type=int, default=20)
     ap.add_argument("--out", default=None)
+    ap.add_argument("--variants", default=None, metavar="LOG2D,M",
+                    help="instead of the sweep, time the calls beside the main path at d = 2^LOG2D with M workers")
     args = ap.parse_args(argv)
     if not torch.cuda.is_available():
         raise SystemExit("the sweep needs a CUDA device")
@@ -115,6 +158,16 @@ def main(argv=None):
     print(header)
     if out:
         out.write(header + "\n")
+    if args.variants:
+        k, M = [int(t) for t in args.variants.split(",")]
+        for r in run_variants(1 << k, M, max(2, args.reps // 4), dev):
+            line = "%d\t%d\t%s\t%.2f\t%.1f\t%.3f\t%d" % r
+            print(line, flush=True)
+            if out:
+                out.write(line + "\n")
+        if out:
+            out.close()
+        return 0
     for M in [int(t) for t in args.workers.split(",")]:
         for k in range(args.min_log2, args.max_log2 + 1):
             reps = args.reps if k < 24 else max(2, args.reps // 8)
