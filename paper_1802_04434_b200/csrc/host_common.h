@@ -56,12 +56,12 @@ ssgd_status launch_status() { return cudaGetLastError() == cudaSuccess ? SSGD_OK
 constexpr unsigned long long kMaxGrid = 0x7FFFFFFFull;
 unsigned grid_for(unsigned long long ctas) { return (unsigned)(ctas < kMaxGrid ? ctas : kMaxGrid); }
 
-// Elements per thread: 4 * unroll.  Large inputs take unroll 4 (eight 128-bit
-// loads in flight per thread in the worker step); smaller ones shrink the tile so
-// that the launch still fills the machine with a few CTAs per SM.
-int pick_unroll(unsigned long long elements_per_row, unsigned long long rows, int sms) {
+// Elements per thread: 4 * unroll.  Large inputs take the largest unroll allowed
+// (eight 128-bit loads in flight per thread in the worker step); smaller ones
+// shrink the tile so that the launch still fills the machine with a few CTAs per SM.
+int pick_unroll(unsigned long long elements_per_row, unsigned long long rows, int sms, int max_unroll = 4) {
   const unsigned long long want = 8ull * sms;                  // CTAs
-  for (int u = 4; u > 1; u /= 2) {
+  for (int u = max_unroll; u > 1; u /= 2) {
     const unsigned long long tile = (unsigned long long)kThreads * 4 * u;
     if (((elements_per_row + tile - 1) / tile) * rows >= want) return u;
   }

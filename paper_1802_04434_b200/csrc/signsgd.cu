@@ -313,7 +313,9 @@ ssgd_status launch_worker(const float* g, float* m, size_t M, size_t d, size_t l
                           uint32_t* bits, size_t ldw, cudaStream_t s) {
   DeviceInfo di;
   if (!device_info(&di)) return SSGD_ERR_CUDA;
-  switch (pick_unroll(d, M, di.sms)) {
+  // without a momentum there is one array to load: twice the elements per thread keep as many loads in flight
+  switch (pick_unroll(d, M, di.sms, MODE == kSignSGD ? 8 : 4)) {
+    case 8: launch_worker_u<kSignSGD, 8>(g, m, M, d, ld, beta, bits, ldw, s); break;
     case 4: launch_worker_u<MODE, 4>(g, m, M, d, ld, beta, bits, ldw, s); break;
     case 2: launch_worker_u<MODE, 2>(g, m, M, d, ld, beta, bits, ldw, s); break;
     default: launch_worker_u<MODE, 1>(g, m, M, d, ld, beta, bits, ldw, s); break;
@@ -378,10 +380,17 @@ ssgd_status launch_fused(const StepArgs& a, cudaStream_t s, bool* launched) {
   if (a.M > (size_t)kFusedMaxWorkers) return SSGD_OK;
   DeviceInfo di;
   if (!device_info(&di)) return SSGD_ERR_CUDA;
-  const int unroll = pick_unroll(a.d, 1, di.sms) >= 2 ? 2 : 1;
+  // Elements per thread and row: 8 with a momentum (two arrays to load: four 128-bit loads in flight),
+  // 16 without (one array), less for short vectors so that the launch still fills the machine.
+  const int want = MODE == kSignSGD ? 4 : 2;
+  const int fit = pick_unroll(a.d, 1, di.sms);
+  const int unroll = fit < want ? fit : want;
   const unsigned long long tile = (unsigned long long)kThreads * 4 * unroll;
   if ((a.d + tile - 1) / tile > kMaxGrid) return SSGD_OK;
-  const bool ok = unroll == 2 ? launch_fused_mu<MODE, 2>(a, s) : launch_fused_mu<MODE, 1>(a, s);
+  bool ok;
+  if (MODE == kSignSGD && unroll == 4) ok = launch_fused_mu<kSignSGD, 4>(a, s);
+  else if (unroll == 2) ok = launch_fused_mu<MODE, 2>(a, s);
+  else ok = launch_fused_mu<MODE, 1>(a, s);
   if (!ok) return SSGD_ERR_SIZE;
   *launched = true;
   return launch_status();

@@ -4,7 +4,8 @@
                                           [--reps 20] [--out sweep.tsv]
 
 For every point and every kernel of the step (worker momentum + pack, majority vote, apply) and for
-the whole step, prints the time per launch, the algorithmic GB/s and its fraction of the measured
+the whole step (and, as a yardstick for the short vote kernel, for a plain device copy of the vote's
+byte volume), prints the time per launch, the algorithmic GB/s and its fraction of the measured
 copy peak.  Launches are replayed from a CUDA graph between two CUDA events.  When
 one launch touches less than twice the L2 size, the launches rotate over several buffer sets so that
 the combined footprint exceeds it (column `cold` = 1); for the smallest sizes that would need more
@@ -89,6 +90,12 @@ def run_point(d: int, M: int, reps: int, dev) -> list:
     rec("momentum_pack", ms, bytes_worker, n_sets_big * bytes_worker >= 2 * L2_BYTES)
     ms = time_launches(lambda s: B.majority_vote(bits[s], M, d, ldw, vote[s]), n_sets, reps)
     rec("majority_vote", ms, bytes_vote, n_sets * bytes_vote >= 2 * L2_BYTES)
+    # reference for the short vote kernel: a plain device copy that moves the same number of bytes
+    half = max(1, int(bytes_vote / 2) // 4)
+    flat = [b.view(-1) for b in bits]
+    if half <= flat[0].numel() and n_sets > 1:
+        ms = time_launches(lambda s: flat[(s + 1) % n_sets][:half].copy_(flat[s][:half]), n_sets, reps)
+        rec("copy_of_vote_bytes", ms, 2.0 * half * 4, n_sets * bytes_vote >= 2 * L2_BYTES)
     ms = time_launches(lambda s: B.sign_apply(x[s], vote[s], d, delta), n_x, reps)
     rec("sign_apply", ms, bytes_apply, n_x * bytes_apply >= 2 * L2_BYTES)
     ms = time_launches(lambda s: B.signsgd_step(x[s % n_x], g[s % n_sets_big], m[s % n_sets_big], M, d, ld, beta,

@@ -1,9 +1,8 @@
 """GPU parity: every entry point of the C ABI against the CPU oracle, element by
 element on the same seeded inputs.
 
-Acceptance (stated by the task's target and derived from the arithmetic): packed
-sign words and vote words bit-exact; m and x within 1 ulp of fp32
-(|diff| <= 1.2e-7 * |value|).  Both sides evaluate the momentum as the same two
+Acceptance bound: packed sign words and vote words bit-exact; m and x within
+1 ulp of fp32 (|diff| <= 1.2e-7 * |value|).  Both sides evaluate the momentum as the same two
 correctly rounded fp32 operations and the apply step as one correctly rounded
 add, so the tests below demand equality of the fp32 bit patterns, which is
 stricter; a sign bit may therefore never differ either.
@@ -299,8 +298,12 @@ def test_config5_sweep_points_full_parity(d, M):
     run_config_full(wl.sweep_point(d, M))
 
 
-@pytest.mark.parametrize("d,M", [(1 << 26, 7), (1 << 28, 3)])
+@pytest.mark.parametrize("d,M", [(1 << 26, 7), (1 << 28, 3), (1 << 28, 31)])
 def test_config5_large_sweep_points_sampled(d, M):
+    free, _ = torch.cuda.mem_get_info()
+    need = 2 * M * d * 4 + 6 * d * 4 + (8 << 30)
+    if free < need:
+        pytest.skip("needs %.0f GB of free device memory" % (need / 2**30))
     sampled_chunk_parity(wl.sweep_point(d, M), n_chunks=16, chunk=1 << 20, seed=d % 1000 + M)
 
 
