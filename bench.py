@@ -3,14 +3,22 @@
 
 One "step" is one pass of the whole hot path -- per-worker momentum update fused
 with 1-bit sign packing, majority vote over the M packed vectors, unpack-and-apply
-to x -- over one batch of synthetic gradients.  The default workload is the
-Resnet-50-sized vector (d = 25,557,056 with per-tensor padding, M = 7 workers,
-Signum beta = 0.9).
+to x -- over one batch of synthetic gradients, issued as ONE call of the step entry
+point.  The default workload is the largest single-GPU configuration: the
+BERT-large-sized vector (d = 335,141,888, M = 16 workers, Signum beta = 0.9, 45 GB
+on the device), which takes the worker + vote + apply kernels; `--workload
+resnet50` (d = 25,557,056, M = 7) takes the single fused kernel.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+                    [--workload bert|resnet50|small|tie|sweep:<d>x<M>] [--seed S]
+                    [--mode shards|workers]
 
-Prints ONE JSON line.  With --impl reference the CPU oracle is timed instead, on
-a bounded slice of the same workload.
+Prints ONE JSON line.  After the timed region a second pass over the same buffers
+takes per-kernel CUDA-event times (`kernels`), the same step is timed end to end
+from host buffers (`e2e`), and the CPU oracle is timed on a bounded sample on one
+thread and on all host cores (`cpu_baseline`, `cpu_baseline_all_cores`).  With
+--impl reference only the CPU oracle is timed.  `--mode workers` runs Algorithm 3
+with one worker per GPU (an all-gather of the sign words between the ranks).
 """
 from __future__ import annotations
 
@@ -30,14 +38,13 @@ UNIT = "params/s"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 
-# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the dominant kernel,
-# from the ncu capture summarised in profiles/; valid only while the kernel source is unchanged.
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per parameter of one launch, from the ncu
+# captures summarised in profiles/ (taken at a reduced d with the same M and kernels; the path is
+# elementwise, so traffic grows in proportion to d).  Valid only while the kernel sources are unchanged.
 NCU_TRAFFIC = {
-    "source_sha256": "02dbe7eb10a46ec6d0b079026d61e5054a950444d468d14358424998f0538bc3",
-    "workload": "resnet50_d25557056_M7",
-    "bytes_per_launch": 1.533647e9 + 792.951296e6,
+    "source_sha256": "",
+    "per_param": {},
 }
-
 
 KERNEL_SOURCES = ("signsgd.cu", "device_common.cuh", "host_common.h")
 
@@ -54,16 +61,14 @@ def kernel_source_digest():
     return h.hexdigest()
 
 
-def ncu_traffic(workload_name: str):
-    if kernel_source_digest() == NCU_TRAFFIC["source_sha256"] and workload_name == NCU_TRAFFIC["workload"]:
-        return NCU_TRAFFIC["bytes_per_launch"]
-    return None
-
-
-def fused_bytes_per_param(M: int, momentum: bool) -> float:
-    """Algorithmic bytes of the fused step kernel: g (+ m read and written) and one sign bit per worker,
-    one voted bit, x read and written.  The separate vote kernel's re-read of the sign words is gone."""
-    return (12.125 if momentum else 4.125) * M + 8.125
+def ncu_traffic(kernel: str, M: int, d: int):
+    """(bytes per launch, note) scaled from the capture, or (None, why)."""
+    if kernel_source_digest() != NCU_TRAFFIC["source_sha256"]:
+        return None, "kernel sources changed since the ncu capture"
+    rec = NCU_TRAFFIC["per_param"].get("%s:M%d" % (kernel, M))
+    if rec is None:
+        return None, "no ncu capture of this kernel at this M"
+    return rec["bytes_per_param"] * d, "scaled by d from the capture at d = %d" % rec["d"]
 
 
 def measured_peak():
@@ -75,26 +80,46 @@ def measured_peak():
         return FALLBACK_HBM_GBS, "fallback"
 
 
-def get_workload(name: str):
+def get_workload(name: str, seed: int = 0):
     from paper_1802_04434_b200 import workloads as wl
     if name == "resnet50":
-        return wl.resnet50_signum()
-    if name == "small":
-        return wl.small_signum()
-    if name == "tie":
-        return wl.tie_zero_stress()
-    if name == "bert":
-        return wl.bert_large_signum()
-    if name.startswith("sweep:"):
+        cfg = wl.resnet50_signum()
+    elif name == "small":
+        cfg = wl.small_signum()
+    elif name == "tie":
+        cfg = wl.tie_zero_stress()
+    elif name == "bert":
+        cfg = wl.bert_large_signum()
+    elif name.startswith("sweep:"):
         d, M = name.split(":")[1].split("x")
-        return wl.sweep_point(int(d), int(M))
-    raise SystemExit("unknown workload %r" % name)
+        cfg = wl.sweep_point(int(d), int(M))
+    else:
+        raise SystemExit("unknown workload %r" % name)
+    cfg.seed = seed
+    return cfg
+
+
+# algorithmic bytes per parameter of each kernel (fp32 state in place, 1 bit per sign)
+def worker_bpp(M: int, momentum: bool) -> float:
+    return (12.125 if momentum else 4.125) * M
+
+
+def vote_bpp(M: int) -> float:
+    return (M + 1) / 8.0
+
+
+APPLY_BPP = 8.125
+
+
+def fused_bpp(M: int, momentum: bool) -> float:
+    """The fused step kernel never reads the sign words back: worker bytes + apply bytes."""
+    return worker_bpp(M, momentum) + APPLY_BPP
 
 
 # ----------------------------------------------------------------------------- clocks
 
 class ClockSampler:
-    """Samples SM clock and clock-event reasons through NVML while the GPU is under load."""
+    """Samples SM clock and clock-event reasons through NVML (read-only) while the GPU is under load."""
     REASONS = {0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x20: "sw_thermal_slowdown",
                0x40: "hw_thermal_slowdown", 0x80: "hw_power_brake_slowdown", 0x2: "applications_clocks_setting",
                0x10: "sync_boost", 0x100: "display_clock_setting"}
@@ -167,51 +192,123 @@ class ClockSampler:
 
 # ----------------------------------------------------------------------------- the oracle arm
 
-def oracle_rate(cfg, n_sample: int, steps: int, warmup: int):
-    """Time the CPU oracle's whole step on the first n_sample elements of the workload."""
+def host_cores() -> int:
+    try:
+        return len(os.sched_getaffinity(0))
+    except AttributeError:
+        return os.cpu_count() or 1
+
+
+def oracle_inputs(cfg, n: int):
+    """Host arrays (x [n], g [M, n], m [M, n] or None) of the first n parameters of the workload.
+
+    Only the sample is drawn, never the whole vector.  The random draws run on the GPU when there is
+    one (same recipe, much faster for the large samples of the all-cores leg), else on the CPU."""
+    import numpy as np
+    import torch
+    sub = cfg.prefix(n // 32 * 32 if n >= 32 else n)
+    n = sub.d
+    dev = "cuda" if torch.cuda.is_available() else "cpu"
+    g = sub.g(0, dev, sub.shared(dev))[:, :n].contiguous().cpu().numpy()
+    x = sub.x0(dev)[:n].contiguous().cpu().numpy()
+    m = np.zeros((cfg.M, n), dtype=np.float32) if cfg.momentum_buffer else None
+    if dev == "cuda":
+        torch.cuda.empty_cache()
+    return x, g, m
+
+
+def oracle_rate(cfg, n_sample: int, steps: int, warmup: int, threads: int = 1):
+    """Time the CPU oracle's whole step, as it stands, on the first n_sample parameters.
+
+    threads == 1: one call per step.  threads > 1: the sample is cut into `threads` contiguous slices
+    with 32-aligned starts and the same oracle function runs on every slice at once from Python threads
+    (ctypes releases the interpreter lock during the call; the oracle itself is untouched).
+    Returns (params/s, seconds per step, parameters per step)."""
     import numpy as np
     import oracle
-    n = min(n_sample, cfg.d)
-    shared = cfg.shared("cpu")
-    g = cfg.g(0, "cpu", shared)[:, :n].contiguous().numpy().reshape(-1)
-    x = cfg.x0("cpu")[:n].contiguous().numpy()
-    m = np.zeros(cfg.M * n, dtype=np.float32) if cfg.momentum_buffer else None
+    x, g, m = oracle_inputs(cfg, min(n_sample, cfg.d))
+    n = x.size
+    M = cfg.M
+    if threads <= 1:
+        gf = g.reshape(-1)
+        mf = None if m is None else m.reshape(-1)
+
+        def one_step():
+            oracle.signsgd_step(x, gf, mf, M, n, cfg.beta, cfg.delta)
+    else:
+        from concurrent.futures import ThreadPoolExecutor
+        per = max(32, (n // threads) // 32 * 32)
+        cuts = [min(n, t * per) for t in range(threads)] + [n]
+        parts = []
+        for a, b in zip(cuts[:-1], cuts[1:]):
+            if b > a:
+                parts.append((np.ascontiguousarray(x[a:b]), np.ascontiguousarray(g[:, a:b]).reshape(-1),
+                              None if m is None else np.ascontiguousarray(m[:, a:b]).reshape(-1), b - a))
+        del x, g, m
+        pool = ThreadPoolExecutor(max_workers=len(parts))
+
+        def run_part(p):
+            oracle.signsgd_step(p[0], p[1], p[2], M, p[3], cfg.beta, cfg.delta)
+
+        def one_step():
+            list(pool.map(run_part, parts))
+        threads = len(parts)
     for _ in range(warmup):
-        oracle.signsgd_step(x, g, m, cfg.M, n, cfg.beta, cfg.delta)
+        one_step()
     t0 = time.perf_counter()
     for _ in range(steps):
-        oracle.signsgd_step(x, g, m, cfg.M, n, cfg.beta, cfg.delta)
+        one_step()
     dt = time.perf_counter() - t0
-    return n * steps / dt, dt / steps, n
+    return n * steps / dt, dt / steps, n, max(threads, 1)
+
+
+ORACLE_SAMPLE_MAX_FLOATS = 1 << 28      # M * n of the sample: 1 GiB of gradients (and as much momentum) at most
+
+
+def oracle_sample_size(cfg, seconds_per_step: float, threads: int = 1, probe=None) -> int:
+    """Parameters per step that keep one oracle step near `seconds_per_step` (3 s at most) and the
+    sample's host buffers bounded."""
+    rate = probe if probe is not None else oracle_rate(cfg, 1 << 17, 1, 1)[0]
+    n = int(rate * min(seconds_per_step, 3.0)) * max(threads, 1)
+    n = min(n, cfg.d, ORACLE_SAMPLE_MAX_FLOATS // cfg.M)
+    return max(1 << 12, n) // 32 * 32
 
 
 def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    cfg = get_workload(args.workload)
-    # size each step's slice so that the whole run stays near a minute of CPU time
-    rate, _, _ = oracle_rate(cfg, 1 << 18, 1, 1)
+    cfg = get_workload(args.workload, args.seed)
+    cores = host_cores()
+    threads = cores if args.ref_threads <= 0 else min(args.ref_threads, cores)
+    # size each step's slice so that the whole run stays near a minute of wall time
     budget_s = 60.0
-    n = int(rate * budget_s / max(args.steps + args.warmup, 1))
-    n = max(1 << 12, min(cfg.d, n)) // 32 * 32
-    value, s_per_step, n = oracle_rate(cfg, n, args.steps, args.warmup)
-    sample = "first %d of %d elements per step, all M=%d workers, single thread" % (n, cfg.d, cfg.M)
+    per_step = budget_s / max(args.steps + args.warmup, 1)
+    n = args.ref_sample if args.ref_sample > 0 else oracle_sample_size(cfg, per_step, threads)
+    value, s_per_step, n, used = oracle_rate(cfg, n, args.steps, args.warmup, threads)
+    sample = ("first %d of %d parameters per step, all M=%d workers, %d thread(s) on disjoint 32-aligned "
+              "slices, unmodified oracle" % (n, cfg.d, cfg.M, used))
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": s_per_step * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
         "data": "synthetic",
-        "config": workload_config(cfg, args.gpus),
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "config": workload_config(cfg, args.gpus, args.mode),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": used, "host_cores": cores, "kind": "oracle",
+                         "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }
     print(json.dumps(line), flush=True)
 
 
-def workload_config(cfg, n_gpus):
-    return {"workload": cfg.name, "d": cfg.d, "M": cfg.M, "beta": cfg.beta, "delta": cfg.delta,
-            "parallelism": "independent shard of d per GPU, no collective" if n_gpus > 1 else "single GPU",
+def workload_config(cfg, n_gpus, mode="shards"):
+    if mode == "workers":
+        par = ("Algorithm 3 with one worker per GPU: M = %d ranks, each packs its own sign row, all-gather of the "
+               "rows, local vote and apply" % n_gpus)
+    else:
+        par = "independent shard of d per GPU, no collective" if n_gpus > 1 else "single GPU"
+    return {"workload": cfg.name, "d": cfg.d, "M": cfg.M if mode != "workers" else n_gpus, "beta": cfg.beta,
+            "delta": cfg.delta, "seed": cfg.seed, "mode": mode, "parallelism": par,
             "l2": "g + m per step exceed L2 (no flush needed)" if not needs_l2_flush(cfg)
             else "L2 flushed between timed steps by writing a 256 MiB buffer; step time = sum of per-step event pairs"}
 
@@ -222,6 +319,109 @@ def needs_l2_flush(cfg) -> bool:
 
 
 # ----------------------------------------------------------------------------- the CUDA arm
+
+class Buffers:
+    """Device state of one workload: x, g, m, the word workspaces."""
+
+    def __init__(self, cfg, dev):
+        import torch
+        self.cfg = cfg
+        shared = cfg.shared(dev)
+        self.x = cfg.x0(dev)
+        self.m = cfg.m0(dev) if cfg.momentum_buffer else None
+        self.g = cfg.g(0, dev, shared)
+        del shared
+        self.bits = torch.zeros(cfg.M, cfg.ldw, dtype=torch.int32, device=dev)
+        self.vote = torch.zeros(cfg.words, dtype=torch.int32, device=dev)
+
+
+def make_step(B, b, stream):
+    cfg = b.cfg
+
+    def step():
+        B.signsgd_step(b.x, b.g, b.m, cfg.M, cfg.d, cfg.ld, cfg.beta, cfg.delta, b.bits, cfg.ldw, b.vote, stream)
+    return step
+
+
+def timed_block(step, K, stream, flush, torch):
+    """K steps between two events; with a flush buffer, each step between its own pair and the flush outside."""
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    if flush is None:
+        t0.record(stream)
+        for _ in range(K):
+            step()
+        t1.record(stream)
+        return lambda: t0.elapsed_time(t1)
+    pairs = []
+    for _ in range(K):
+        a, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        step()
+        e.record(stream)
+        flush.zero_()
+        pairs.append((a, e))
+    return lambda: sum(a.elapsed_time(e) for a, e in pairs)
+
+
+def per_kernel_pass(B, b, K, stream, flush, torch):
+    """Second pass over the same buffers: CUDA-event pairs around every kernel of the step.
+
+    For M <= FUSED_MAX_WORKERS the step is one fused kernel; otherwise the three entry points the step
+    entry point issues are called one by one so that events can sit between the kernels."""
+    cfg = b.cfg
+    M, d, ld, ldw = cfg.M, cfg.d, cfg.ld, cfg.ldw
+    momentum = cfg.momentum_buffer
+    fused = M <= B.FUSED_MAX_WORKERS
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    marks = []
+    for _ in range(K):
+        e = [ev()]
+        e[0].record(stream)
+        if fused:
+            B.signsgd_step(b.x, b.g, b.m, M, d, ld, cfg.beta, cfg.delta, b.bits, ldw, b.vote, stream)
+            e.append(ev()); e[-1].record(stream)
+        else:
+            if momentum:
+                B.signum_momentum_pack(b.g, b.m, M, d, ld, cfg.beta, b.bits, ldw, stream)
+            else:
+                B.sign_pack(b.g, M, d, ld, b.bits, ldw, stream)
+            e.append(ev()); e[-1].record(stream)
+            B.majority_vote(b.bits, M, d, ldw, b.vote, stream)
+            e.append(ev()); e[-1].record(stream)
+            B.sign_apply(b.x, b.vote, d, cfg.delta, stream)
+            e.append(ev()); e[-1].record(stream)
+        if flush is not None:
+            flush.zero_()
+        marks.append(e)
+    torch.cuda.synchronize()
+    n = len(marks[0]) - 1
+    ms = [sum(e[i].elapsed_time(e[i + 1]) for e in marks) / K for i in range(n)]
+    if fused:
+        names = [("fused_step_kernel", "ssgd_signsgd_step", fused_bpp(M, momentum))]
+    else:
+        names = [("worker_pack_kernel", "ssgd_signum_momentum_pack" if momentum else "ssgd_sign_pack",
+                  worker_bpp(M, momentum)),
+                 ("vote_kernel", "ssgd_majority_vote", vote_bpp(M)),
+                 ("apply_kernel", "ssgd_sign_apply", APPLY_BPP)]
+    return [(k, ep, bpp, t) for (k, ep, bpp), t in zip(names, ms)]
+
+
+def kernel_entry(kernel, entry_point, bpp, ms, cfg, peak, launches):
+    gbs = bpp * cfg.d / (ms * 1e-3) / 1e9
+    traffic, note = ncu_traffic(kernel, cfg.M, cfg.d)
+    return {"kernel": kernel, "entry_point": entry_point, "workload": cfg.name, "M": cfg.M,
+            "bytes_per_param": bpp, "units_per_launch": cfg.d, "bytes_per_launch": bpp * cfg.d,
+            "launches_timed": launches, "ms_per_launch": ms, "achieved_gbs": gbs, "frac": gbs / peak,
+            "frac_of_nominal_8TBs": gbs / NOMINAL_HBM_GBS, "traffic": traffic, "traffic_note": note}
+
+
+def host_buffer(torch, shape, dtype):
+    """Page-locked host tensor if the box grants it, else pageable; returns (tensor, kind)."""
+    try:
+        return torch.empty(shape, dtype=dtype, pin_memory=True), "pinned"
+    except Exception:
+        return torch.empty(shape, dtype=dtype), "pageable"
+
 
 def run_ours(args):
     import torch
@@ -235,134 +435,203 @@ def run_ours(args):
     dev = torch.device("cuda", local_rank)
     multi.init(dev)
     B.lib()  # fail here, loudly, if the CUDA library is missing
+    if args.mode == "workers":
+        return run_workers(args, torch, B, multi, dev, rank, local_rank, world)
 
-    cfg = get_workload(args.workload)
-    cfg.seed = multi.shard_seed(rank)   # every rank owns an independent shard of a larger vector
+    cfg = get_workload(args.workload, args.seed + multi.shard_seed(rank))  # an independent shard per rank
     M, d, ld, ldw, W = cfg.M, cfg.d, cfg.ld, cfg.ldw, cfg.words
     momentum = cfg.momentum_buffer
-    shared = cfg.shared(dev)
-    x = cfg.x0(dev)
-    m = cfg.m0(dev) if momentum else None
-    g = cfg.g(0, dev, shared)
-    del shared
-    bits = torch.zeros(M, ldw, dtype=torch.int32, device=dev)
-    vote = torch.zeros(W, dtype=torch.int32, device=dev)
+    free, _ = torch.cuda.mem_get_info()
+    need = (2 if momentum else 1) * M * ld * 4 + 4 * d * 4 + (2 << 30)
+    if free < need:
+        raise SystemExit("workload %s needs %.1f GB of device memory, %.1f GB are free" % (cfg.name, need / 1e9, free / 1e9))
+    b = Buffers(cfg, dev)
     stream = torch.cuda.current_stream()
-
+    step = make_step(B, b, stream)
     fused = M <= B.FUSED_MAX_WORKERS
-
-    def step_with_events(ev):
-        # With few workers one step is one call of the step entry point = one fused kernel launch, and
-        # the event pair around it times that kernel.  With more workers the step entry point issues the
-        # worker, vote and apply kernels; the same three entry points are then called here one by one so
-        # that the event pair can sit around the dominant (worker) kernel inside the timed region.
-        ev[0].record(stream)
-        if fused:
-            B.signsgd_step(x, g, m, M, d, ld, cfg.beta, cfg.delta, bits, ldw, vote, stream)
-            ev[1].record(stream)
-            return
-        if momentum:
-            B.signum_momentum_pack(g, m, M, d, ld, cfg.beta, bits, ldw, stream)
-        else:
-            B.sign_pack(g, M, d, ld, bits, ldw, stream)
-        ev[1].record(stream)
-        B.majority_vote(bits, M, d, ldw, vote, stream)
-        B.sign_apply(x, vote, d, cfg.delta, stream)
-
-    def barrier():
-        multi.barrier(dev)
-
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev) if needs_l2_flush(cfg) else None
     K, Wm = args.steps, args.warmup
-    events = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
-    scratch_ev = (torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
-    for _ in range(Wm):
-        step_with_events(scratch_ev)
-    sampler = ClockSampler(local_rank)
-    t_start, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
-    sampler.start()
-    t_start.record(stream)
-    step_ends = []
-    for k in range(K):
-        step_with_events(events[k])
-        if flush is not None:
-            e = torch.cuda.Event(enable_timing=True)
-            e.record(stream)
-            step_ends.append(e)
-            flush.zero_()
-    t_end.record(stream)
-    barrier()
-    sampler.stop()
-    elapsed_ms = t_start.elapsed_time(t_end)
-    if flush is not None:       # leave the flush writes out: each step from its first event to its own end
-        elapsed_ms = sum(events[k][0].elapsed_time(step_ends[k]) for k in range(K))
-    clock_note = None
-    if sampler.ok and len(sampler.samples) < 5:
-        # timed region too short for the sampling period: keep sampling under the same load
-        clock_note = "timed region shorter than 5 sampling periods; sampled under the same load right after it"
-        sampler.start()
-        t0 = time.perf_counter()
-        while time.perf_counter() - t0 < 0.5:
-            for _ in range(20):
-                step_with_events(scratch_ev)
-            torch.cuda.synchronize()
-        sampler.stop()
-    worker_ms = sum(a.elapsed_time(b) for a, b in events) / K
 
-    elapsed_ms, worker_ms = multi.max_over_ranks([elapsed_ms, worker_ms], dev)
+    for _ in range(Wm):
+        step()
+    sampler = ClockSampler(local_rank)
+    multi.barrier(dev)
+    sampler.start()
+    read_ms = timed_block(step, K, stream, flush, torch)
+    multi.barrier(dev)
+    elapsed_ms = read_ms()
+    # The clock samples must be of timed work: when the K steps end before five sampling periods have
+    # passed, the same K-step block is repeated (each block timed the same way) until they have.
+    extra = []
+    while sampler.ok and len(sampler.samples) < 5 and len(extra) < 2000:
+        r = timed_block(step, K, stream, flush, torch)
+        torch.cuda.synchronize(dev)
+        extra.append(r())
+    sampler.stop()
+    clock_note = None
+    if extra:
+        clock_note = ("the %d-step block was repeated %d more times inside the sampling window (median block "
+                      "%.4f ms); value is the first block's" % (K, len(extra), sorted(extra)[len(extra) // 2]))
+
+    kernels = per_kernel_pass(B, b, K, stream, flush, torch)
+    (elapsed_ms, *kms) = multi.max_over_ranks([elapsed_ms] + [t for *_, t in kernels], dev)
+    kernels = [(k, ep, bpp, t) for (k, ep, bpp, _), t in zip(kernels, kms)]
     value = multi.whole_job_rate(d, K, elapsed_ms, world)
     ms_per_step = elapsed_ms / K
 
-    # end to end through the host-buffer entry point: gradients start in pinned host memory,
-    # the voted words come back to the host, every step
-    Ke = max(3, min(K, args.e2e_steps))
-    g_host = torch.empty(M, ld, dtype=torch.float32).pin_memory()
-    g_host.copy_(g)
-    vote_host = torch.zeros(W, dtype=torch.int32).pin_memory()
-    for _ in range(3):
-        B.signsgd_step_host(x, g_host, m, M, d, ld, cfg.beta, cfg.delta, g, bits, ldw, vote, vote_host, stream)
-    barrier()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record(stream)
-    for _ in range(Ke):
-        B.signsgd_step_host(x, g_host, m, M, d, ld, cfg.beta, cfg.delta, g, bits, ldw, vote, vote_host, stream)
-    e1.record(stream)
-    barrier()
-    e2e_ms = e0.elapsed_time(e1)
-    (e2e_ms,) = multi.max_over_ranks([e2e_ms], dev)
-    e2e_value = multi.whole_job_rate(d, Ke, e2e_ms, world)
+    # end to end through the host-buffer entry point: every step copies that step's gradients from host
+    # memory to the device, runs the step and copies the voted words back to the host
+    Ke = max(1, min(K, args.e2e_steps))
+    e2e = None
+    try:
+        g_host, host_kind = host_buffer(torch, (M, ld), torch.float32)
+        g_host.copy_(b.g)
+        vote_host, _ = host_buffer(torch, (W,), torch.int32)
+        host_step = lambda: B.signsgd_step_host(b.x, g_host, b.m, M, d, ld, cfg.beta, cfg.delta, b.g, b.bits, ldw,
+                                                b.vote, vote_host, stream)
+        for _ in range(max(1, min(3, args.e2e_warmup))):
+            host_step()
+        multi.barrier(dev)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(Ke):
+            host_step()
+        e1.record(stream)
+        multi.barrier(dev)
+        (e2e_ms,) = multi.max_over_ranks([e0.elapsed_time(e1)], dev)
+        e2e = {"value": multi.whole_job_rate(d, Ke, e2e_ms, world), "unit": UNIT, "h2d_bytes_per_step": M * ld * 4,
+               "d2h_bytes_per_step": W * 4, "steps": Ke, "ms_per_step": e2e_ms / Ke, "host_memory": host_kind,
+               "entry_point": "ssgd_signsgd_step_host",
+               "h2d_gbs": M * ld * 4 / (e2e_ms / Ke * 1e-3) / 1e9}
+        del g_host, vote_host
+    except (RuntimeError, MemoryError) as exc:   # the host could not hold one step's gradients
+        e2e = {"value": None, "unit": UNIT, "h2d_bytes_per_step": M * ld * 4, "d2h_bytes_per_step": W * 4,
+               "error": "host buffer of %.1f GB not granted: %s" % (M * ld * 4 / 1e9, str(exc)[:120])}
+        multi.barrier(dev)
 
+    if rank != 0:
+        multi.finish()
+        return
+    peak, peak_kind = measured_peak()
+    step_bpp = fused_bpp(M, momentum) if fused else worker_bpp(M, momentum) + vote_bpp(M) + APPLY_BPP
+    entries = [kernel_entry(k, ep, bpp, t, cfg, peak, K) for k, ep, bpp, t in kernels]
+    dom = max(entries, key=lambda e: e["ms_per_launch"])
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic",
+        "config": workload_config(cfg, world),
+        "entry_point": "ssgd_signsgd_step",
+        "step_bytes_per_param": step_bpp,
+        "step_hbm_gbs": step_bpp * d / (ms_per_step * 1e-3) / 1e9,
+        "step_frac_of_nominal_8TBs": step_bpp * d / (ms_per_step * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
+        "roofline": {"kernel": dom["kernel"], "bound": "hbm", "achieved": dom["achieved_gbs"], "peak": peak,
+                     "peak_kind": "of " + peak_kind, "unit": "GB/s", "frac": dom["frac"],
+                     "frac_of_nominal_8TBs": dom["frac_of_nominal_8TBs"], "ms_per_launch": dom["ms_per_launch"],
+                     "bytes_per_launch": dom["bytes_per_launch"], "traffic": dom["traffic"],
+                     "traffic_note": dom["traffic_note"],
+                     "timed_in": "second pass over the same buffers right after the timed region, %d launches, "
+                                 "CUDA events around each kernel" % K},
+        "kernels": entries,
+        "kernels_sum_ms": sum(e["ms_per_launch"] for e in entries),
+        "e2e": e2e,
+        "gpu_launches": K * len(entries),
+        "clocks": sampler.summary(clock_note),
+    }
+    if world == 1 and not args.no_extra_kernels and not fused:
+        # the fused kernel (the path for M <= 8) as one more entry, on the Resnet-50-sized workload
+        del b, step
+        torch.cuda.empty_cache()
+        cfg2 = get_workload("resnet50", args.seed)
+        b2 = Buffers(cfg2, dev)
+        step2 = make_step(B, b2, stream)
+        for _ in range(max(3, Wm)):
+            step2()
+        k2 = per_kernel_pass(B, b2, max(K, 20), stream, None, torch)
+        line["kernels"] += [kernel_entry(k, ep, bpp, t, cfg2, peak, max(K, 20)) for k, ep, bpp, t in k2]
+        del b2, step2
+        torch.cuda.empty_cache()
+    if not args.no_cpu_baseline and world == 1:
+        probe = oracle_rate(cfg, 1 << 17, 1, 1)[0]
+        v, _, n, _ = oracle_rate(cfg, oracle_sample_size(cfg, 3.0, 1, probe), 3, 1)
+        cores = host_cores()
+        line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": 1, "host_cores": cores, "kind": "oracle",
+                                "sample": "first %d of %d parameters, M=%d, 3 steps, one thread" % (n, d, M)}
+        va, _, na, used = oracle_rate(cfg, oracle_sample_size(cfg, 2.0, cores, probe), 3, 1, cores)
+        line["cpu_baseline_all_cores"] = {
+            "value": va, "unit": UNIT, "cores": used, "host_cores": cores, "kind": "oracle",
+            "sample": "first %d of %d parameters, M=%d, 3 steps, %d threads on disjoint 32-aligned slices, "
+                      "unmodified oracle" % (na, d, M, used)}
+    print(json.dumps(line), flush=True)
+    multi.finish()
+
+
+def run_workers(args, torch, B, multi, dev, rank, local_rank, world):
+    """Algorithm 3 with one worker per GPU: rank r is worker r, M = world size."""
+    cfg = get_workload(args.workload, args.seed)
+    d, ld, ldw, W = cfg.d, cfg.ld, cfg.ldw, cfg.words
+    momentum = cfg.momentum_buffer
+    one = cfg.prefix(d)
+    one.M = 1
+    one.seed = args.seed * 1000003 + rank            # every worker draws its own gradient noise
+    shared = cfg.shared(dev)                         # ... around the same mean
+    x = cfg.x0(dev)                                  # replicas of x start (and stay) identical
+    g = one.g(0, dev, shared)
+    m = one.m0(dev) if momentum else None
+    del shared
+    ws = multi.WorkerStep(d, dev)
+    stream = torch.cuda.current_stream()
+    K, Wm = args.steps, args.warmup
+    step = lambda ev=None: ws.step(x, g, m, cfg.beta, cfg.delta, events=ev)
+    for _ in range(Wm):
+        step()
+    sampler = ClockSampler(local_rank)
+    multi.barrier(dev)
+    sampler.start()
+    marks = []
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record(stream)
+    for _ in range(K):
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+        step(ev)
+        marks.append(ev)
+    t1.record(stream)
+    multi.barrier(dev)
+    sampler.stop()
+    elapsed_ms = t0.elapsed_time(t1)
+    pack_ms = sum(e[0].elapsed_time(e[1]) for e in marks) / K
+    xchg_ms = sum(e[1].elapsed_time(e[2]) for e in marks) / K
+    rest_ms = sum(e[2].elapsed_time(e[3]) for e in marks) / K
+    elapsed_ms, pack_ms, xchg_ms, rest_ms = multi.max_over_ranks([elapsed_ms, pack_ms, xchg_ms, rest_ms], dev)
+    same = multi.all_ranks_equal(ws.vote)
     if rank == 0:
         peak, peak_kind = measured_peak()
-        bpp = fused_bytes_per_param(M, momentum) + (0.0 if fused else (M + 1) / 8.0 - 0.125)
-        wbytes = (fused_bytes_per_param(M, momentum) if fused else (12.125 if momentum else 4.125) * M) * d
-        achieved = wbytes / (worker_ms * 1e-3) / 1e9
+        Mw = world
+        pack_bytes = worker_bpp(1, momentum) * d
         line = {
-            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
-            "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "f32", "data": "synthetic",
-            "config": workload_config(cfg, world),
-            "step_hbm_gbs": bpp * d / (ms_per_step * 1e-3) / 1e9,
-            "step_frac_of_nominal_8TBs": bpp * d / (ms_per_step * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
-            "step_bytes_per_param": bpp,
-            "roofline": {"kernel": "fused_step_kernel (momentum + sign + pack, vote, apply)" if fused else
-                         "worker_pack_kernel (momentum + sign + pack)", "bound": "hbm", "achieved": achieved, "peak": peak,
-                         "peak_kind": "of " + peak_kind, "unit": "GB/s", "frac": achieved / peak,
-                         "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
-                         "ms_per_launch": worker_ms, "bytes_per_launch": wbytes,
-                         "traffic": ncu_traffic(cfg.name)},
-            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": M * ld * 4,
-                    "d2h_bytes_per_step": W * 4, "steps": Ke, "ms_per_step": e2e_ms / Ke},
-            "gpu_launches": K if fused else 3 * K,
-            "clocks": sampler.summary(clock_note),
+            "metric": METRIC, "value": d * K / (elapsed_ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K,
+            "warmup": Wm, "ms_per_step": elapsed_ms / K, "higher_is_better": True, "scaling": "strong",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": workload_config(cfg, world, "workers"),
+            "wire_bits_per_step_table1": 2 * Mw * d,
+            "wire_bytes_sent_per_rank_per_step": ws.ldw * 4 * (world - 1),
+            "exchange": {"collective": "all_gather_into_tensor of ceil(d/32)-word rows (NCCL)", "ms": xchg_ms,
+                         "share_of_step": xchg_ms / (elapsed_ms / K)},
+            "kernels": [
+                {"kernel": "worker_pack_kernel", "ms_per_launch": pack_ms, "bytes_per_launch": pack_bytes,
+                 "achieved_gbs": pack_bytes / (pack_ms * 1e-3) / 1e9,
+                 "frac": pack_bytes / (pack_ms * 1e-3) / 1e9 / peak},
+                {"kernel": "vote_kernel + apply_kernel", "ms_per_launch": rest_ms,
+                 "bytes_per_launch": (vote_bpp(Mw) + APPLY_BPP) * d,
+                 "achieved_gbs": (vote_bpp(Mw) + APPLY_BPP) * d / (rest_ms * 1e-3) / 1e9,
+                 "frac": (vote_bpp(Mw) + APPLY_BPP) * d / (rest_ms * 1e-3) / 1e9 / peak}],
+            "roofline": {"kernel": "worker_pack_kernel", "bound": "hbm",
+                         "achieved": pack_bytes / (pack_ms * 1e-3) / 1e9, "peak": peak, "peak_kind": "of " + peak_kind,
+                         "unit": "GB/s", "frac": pack_bytes / (pack_ms * 1e-3) / 1e9 / peak, "traffic": None},
+            "votes_identical_on_all_ranks": bool(same),
+            "gpu_launches": 3 * K,
+            "clocks": sampler.summary(),
         }
-        if not args.no_cpu_baseline and world == 1:
-            rate, _, _ = oracle_rate(cfg, 1 << 18, 1, 1)
-            n = max(1 << 16, min(cfg.d, int(rate * 4.0))) // 32 * 32      # ~4 s per step, 3 timed steps
-            v, _, n = oracle_rate(cfg, n, 3, 1)
-            line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle",
-                                    "sample": "first %d of %d elements, M=%d, 3 steps, single thread" % (n, d, M)}
         print(json.dumps(line), flush=True)
     multi.finish()
 
@@ -370,13 +639,23 @@ def run_ours(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=2000)
-    ap.add_argument("--warmup", type=int, default=50)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
-    ap.add_argument("--workload", default="resnet50",
-                    help="resnet50 | small | tie | bert | sweep:<d>x<M>")
-    ap.add_argument("--e2e-steps", type=int, default=40)
+    ap.add_argument("--workload", default="bert",
+                    help="bert (default, the largest single-GPU configuration) | resnet50 | small | tie | sweep:<d>x<M>")
+    ap.add_argument("--mode", choices=["shards", "workers"], default="shards",
+                    help="shards: every GPU simulates all M workers on its own shard of parameters (no collective); "
+                         "workers: one worker per GPU, sign rows all-gathered (Algorithm 3 as a distributed step)")
+    ap.add_argument("--seed", type=int, default=0)
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--e2e-warmup", type=int, default=1)
+    ap.add_argument("--ref-threads", type=int, default=0, help="threads of the oracle arm (0 = all host cores)")
+    ap.add_argument("--ref-sample", type=int, default=0,
+                    help="parameters per step of the oracle arm (0 = sized from a probe of its speed)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-extra-kernels", action="store_true",
+                    help="skip the extra fused-kernel entry on the Resnet-50-sized workload")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3

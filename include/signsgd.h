@@ -121,9 +121,9 @@ ssgd_status ssgd_signsgd_step(float* x, const float* g, float* m, size_t M,
  * beta is outside [0,1) or NaN.  The scan takes about 5/(1-beta) iterations. */
 size_t ssgd_warmup_steps(float beta);
 
-/* Theorem 3's warm-up iteration on the worker side: "accumulate the momentum as
- * normal, but use the sign of the stochastic gradient to make updates".  Same as
- * ssgd_signum_momentum_pack (m updated in place, identical values) except that
+/* Theorem 3's warm-up iteration on the worker side: the momentum is updated as
+ * in Algorithm 2, but the bit sent is the sign of the stochastic gradient.  Same
+ * as ssgd_signum_momentum_pack (m updated in place, identical values) except that
  * bit i of row w = !(g[w][i] < 0), the words of ssgd_sign_pack.               */
 ssgd_status ssgd_signum_warmup_pack(const float* g, float* m, size_t M, size_t d,
                                     size_t ld, float beta, uint32_t* bits,
@@ -176,7 +176,7 @@ ssgd_status ssgd_ternary_pack(const float* g, float* m, size_t M, size_t d, size
 
 /* Server side: with P / N the numbers of active +1 / -1 votes on a parameter, the
  * answer is sign(P - N) when |P - N| >= max(quorum, 1) ("quorum reached") and 0
- * otherwise (too many workers disagreed or abstained; a tie never decides).
+ * otherwise (the margin among the cast votes is too small; a tie never decides).
  *   vote_active out [W]: bit set = a decision was taken;
  *   vote_sign   out [W]: bit set = decided +1 (0 where undecided).             */
 ssgd_status ssgd_quorum_vote(const uint32_t* sign_bits, const uint32_t* active_bits,
@@ -254,14 +254,18 @@ ssgd_status ssgd_signsgd_step_host(float* x, const float* g_host, float* m,
  *   DEVICE pointers with the same rules as ssgd_signsgd_step.
  *
  * The first call on each device looks up the device address of the built-in
- * array (with that device current) and remembers it; make that first call before
- * starting any stream capture.  All calls on a device share the one array, and it
- * keeps whatever the previous call left there; nothing in it has to start at
- * zero, because every word the step reads back it has written first.  Two calls
- * whose GPU work can overlap (different streams, or different host threads on the
- * same device) race on that array: issue them on one stream, or order them
- * yourself.  The wire words are not returned; callers who want them use
- * ssgd_signsgd_step. */
+ * array (with that device current) and remembers it for as long as the device's
+ * primary context lives (after cudaDeviceReset the remembered address is stale:
+ * do not call this again in that process); make that first call before starting
+ * any stream capture.  All calls on a device share the one array, and it keeps
+ * whatever the previous call left there.  Nothing in it has to start at zero:
+ * every sign word and vote word that can reach x is written by the call before
+ * it is read; the only stale words a call may read are the up to three padding
+ * words that round a row up to a multiple of 4, and the vote masks every bit at
+ * a position >= d, so they cannot influence any output bit.  Two calls whose GPU
+ * work can overlap (different streams, or different host threads on the same
+ * device) race on that array: issue them on one stream, or order them yourself.
+ * The wire words are not returned; callers who want them use ssgd_signsgd_step. */
 ssgd_status ssgd_signsgd_step_noalloc(float* x, const float* g, float* m,
                                       size_t M, size_t d, size_t ld, float beta,
                                       float delta, void* stream);

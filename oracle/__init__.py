@@ -49,6 +49,8 @@ def _load():
     L.ssgd_words_ref.argtypes = [sz]
     L.ssgd_density_ref.restype = ctypes.c_double
     L.ssgd_density_ref.argtypes = [vp, sz, vp, vp]
+    L.ssgd_density_of_root_ref.restype = ctypes.c_double
+    L.ssgd_density_of_root_ref.argtypes = [vp, sz, vp, vp]
     L.ssgd_count_planes_ref.restype = sz
     L.ssgd_count_planes_ref.argtypes = [sz]
     L.ssgd_warmup_steps_ref.restype = sz
@@ -288,6 +290,15 @@ def density(v: np.ndarray):
     l1, l2 = ctypes.c_double(), ctypes.c_double()
     phi = _load().ssgd_density_ref(_chk(v, np.float32, v.size, "v"), v.size, ctypes.addressof(l1),
                                    ctypes.addressof(l2))
+    return float(phi), l1.value, l2.value
+
+
+def density_of_root(v: np.ndarray):
+    """phi(sqrt(v)) for a non-negative v (Sec. 3: the noise density from a vector of variances);
+    returns (phi, sum sqrt(v_i), sum v_i)."""
+    l1, l2 = ctypes.c_double(), ctypes.c_double()
+    phi = _load().ssgd_density_of_root_ref(_chk(v, np.float32, v.size, "v"), v.size, ctypes.addressof(l1),
+                                           ctypes.addressof(l2))
     return float(phi), l1.value, l2.value
 
 

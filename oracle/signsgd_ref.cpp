@@ -212,10 +212,9 @@ void ssgd_sum_apply_ref(float* x, const uint32_t* counts, size_t M, size_t d,
 }
 
 // ---- majority vote with abstention (Discussion section) ------------------------
-// The paper states the scheme in words: a worker sends its vote "unless [it is]
-// very unsure about the sign of the true gradient in which case [it] send[s]
-// zero"; the server "counts the votes, and if quorum is not reached (i.e. too many
-// workers disagreed or abstained) [it] sends back zero".  No thresholds are given,
+// The paper gives the scheme in words only (Discussion section): a worker that
+// doubts the sign of the true gradient sends 0 instead of +-1, and the server
+// answers 0 when the cast votes do not reach a quorum.  No thresholds are given,
 // so the two used here are a definition of this code base, not the paper's:
 // a worker is unsure when |v| < tau; quorum is reached when |P - N| >= max(Q, 1),
 // P / N being the numbers of +1 / -1 votes cast.  (Parity with the paper is
@@ -281,6 +280,22 @@ double ssgd_density_ref(const float* v, size_t d, double* l1_out, double* l2sq_o
   for (size_t i = 0; i < d; ++i) {
     l1 += std::fabs((double)v[i]);
     l2sq += (double)v[i] * (double)v[i];
+  }
+  if (l1_out) *l1_out = l1;
+  if (l2sq_out) *l2sq_out = l2sq;
+  if (d == 0 || !(l2sq > 0.0)) return 0.0;
+  return l1 * l1 / ((double)d * l2sq);
+}
+
+// Density of the element-wise square root of a non-negative vector, phi(sqrt(v)):
+// Section 3 measures phi(sigma) of the noise vector sigma, whose squares (the
+// per-component variances, up to a common factor that cancels in phi) are what a
+// variance estimator holds.  |sqrt(v)|_1 = sum sqrt(v_i), |sqrt(v)|_2^2 = sum v_i.
+double ssgd_density_of_root_ref(const float* v, size_t d, double* l1_out, double* l2sq_out) {
+  double l1 = 0.0, l2sq = 0.0;
+  for (size_t i = 0; i < d; ++i) {
+    l1 += std::sqrt((double)v[i]);
+    l2sq += (double)v[i];
   }
   if (l1_out) *l1_out = l1;
   if (l2sq_out) *l2sq_out = l2sq;

@@ -19,15 +19,15 @@ struct DeviceInfo {
 bool device_info(DeviceInfo* out) {
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return false;
-  static int cached_sms[64] = {0};
+  static int cached_sms[64] = {0};   // filled on first use; any thread stores the same value
   if (dev < 0 || dev >= 64) return false;
-  if (cached_sms[dev] == 0) {
-    int sms = 0;
+  int sms = __atomic_load_n(&cached_sms[dev], __ATOMIC_RELAXED);
+  if (sms == 0) {
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
       return false;
-    cached_sms[dev] = sms;
+    __atomic_store_n(&cached_sms[dev], sms, __ATOMIC_RELAXED);
   }
-  out->sms = cached_sms[dev];
+  out->sms = sms;
   return true;
 }
 

@@ -129,6 +129,16 @@ class Workload:
     def shared(self, device="cpu"):
         return None if self._shared is None else self._shared(self, device)
 
+    def prefix(self, n: int) -> "Workload":
+        """The same recipe on a vector of the first min(n, d) parameters: same seeds, same per-tensor
+        layout (tensors beyond n dropped, the one that straddles n cut short).  For callers that want a
+        bounded sample of a large workload without drawing all of it."""
+        n = min(int(n), self.d)
+        segs = None
+        if self.segments is not None:
+            segs = [(off, min(size, n - off)) for off, size in self.segments if off < n]
+        return dataclasses.replace(self, d=n, segments=segs)
+
     def g(self, step: int, device="cpu", shared=None, out: Optional[torch.Tensor] = None) -> torch.Tensor:
         """Gradients of all M workers at `step`, shape [M, ld]."""
         if shared is None:

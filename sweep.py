@@ -1,7 +1,7 @@
 """Per-kernel bandwidth sweep: d = 2^10 .. 2^28, M in {1, 3, 7, 15, 31}, Signum beta = 0.9.
 
-    python -m paper_1802_04434_b200.sweep [--min-log2 10] [--max-log2 28] [--workers 1,3,7,15,31]
-                                          [--reps 20] [--out sweep.tsv]
+    python sweep.py [--min-log2 10] [--max-log2 28] [--workers 1,3,7,15,31]
+                    [--reps 20] [--out sweep.tsv]
 
 For every point and every kernel of the step (worker momentum + pack, majority vote, apply) and for
 the whole step (and, as a yardstick for the short vote kernel, for a plain device copy of the vote's
@@ -18,16 +18,20 @@ import json
 import os
 import sys
 
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
 import torch
 
-from . import binding as B
+from paper_1802_04434_b200 import binding as B
 
 L2_BYTES = 126 << 20
 MAX_SETS = 48
 
 
 def peak_gbs() -> float:
-    p = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "MEASURED_PEAKS.json")
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     try:
         with open(p) as fh:
             return float(json.load(fh)["hbm_gbs"])
@@ -90,12 +94,16 @@ def run_point(d: int, M: int, reps: int, dev) -> list:
     rec("momentum_pack", ms, bytes_worker, n_sets_big * bytes_worker >= 2 * L2_BYTES)
     ms = time_launches(lambda s: B.majority_vote(bits[s], M, d, ldw, vote[s]), n_sets, reps)
     rec("majority_vote", ms, bytes_vote, n_sets * bytes_vote >= 2 * L2_BYTES)
-    # reference for the short vote kernel: a plain device copy that moves the same number of bytes
+    # yardstick for the short vote kernel: a plain device copy that moves the same number of bytes.
+    # Sources and destinations are separate buffers and both rotate, so no launch reads what an
+    # earlier one left in L2.
     half = max(1, int(bytes_vote / 2) // 4)
-    flat = [b.view(-1) for b in bits]
-    if half <= flat[0].numel() and n_sets > 1:
-        ms = time_launches(lambda s: flat[(s + 1) % n_sets][:half].copy_(flat[s][:half]), n_sets, reps)
-        rec("copy_of_vote_bytes", ms, 2.0 * half * 4, n_sets * bytes_vote >= 2 * L2_BYTES)
+    if n_sets > 1:
+        src = [torch.randint(0, 1 << 30, (half,), dtype=torch.int32, device=dev) for _ in range(2 * n_sets)]
+        dst = [torch.empty(half, dtype=torch.int32, device=dev) for _ in range(2 * n_sets)]
+        ms = time_launches(lambda s: dst[s].copy_(src[s]), 2 * n_sets, reps)
+        rec("copy_of_vote_bytes", ms, 2.0 * half * 4, 2 * n_sets * half * 4 >= 2 * L2_BYTES)
+        del src, dst
     ms = time_launches(lambda s: B.sign_apply(x[s], vote[s], d, delta), n_x, reps)
     rec("sign_apply", ms, bytes_apply, n_x * bytes_apply >= 2 * L2_BYTES)
     ms = time_launches(lambda s: B.signsgd_step(x[s % n_x], g[s % n_sets_big], m[s % n_sets_big], M, d, ld, beta,

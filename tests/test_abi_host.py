@@ -108,8 +108,18 @@ def test_step_argument_checks(L):
     assert h(A, A, A, 1, 64, 64, 0.9, 0.1, A + 4, A, 4, A, None, None) == ALIGN
 
 
+def test_noalloc_step_rejects_before_touching_the_device(L):
+    # capacity and range checks come before the first CUDA call, so fake pointers are safe here
+    f = L.ssgd_signsgd_step_noalloc
+    assert f(A, A, A, 0, 64, 64, 0.9, 0.1, None) == SIZE
+    assert f(A, A, A, 1025, 64, 64, 0.9, 0.1, None) == SIZE
+    assert f(A, A, A, 7, 1 << 25, 1 << 25, 0.9, 0.1, None) == 6           # (7 + 1) * 2^20 words > 4 Mi
+    assert f(A, A, A, 3, 32 * (1 << 20) + 1, 32 * (1 << 20) + 4, 0.9, 0.1, None) == 6
+    assert b"scratch" in L.ssgd_status_str(6)
+
+
 def test_warmup_steps_is_host_arithmetic(L):
-    assert L.ssgd_warmup_steps(0.9) == 54          # Theorem 3: "for beta = 0.9 we have C = 54"
+    assert L.ssgd_warmup_steps(0.9) == 54          # the value Theorem 3 prints for beta = 0.9
     assert L.ssgd_warmup_steps(0.0) == 1
     assert L.ssgd_warmup_steps(1.0) == 0 and L.ssgd_warmup_steps(float("nan")) == 0
     w = L.ssgd_signsgd_warmup_step

@@ -9,7 +9,8 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 def test_reference_arm_prints_one_json_line():
     out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--steps", "2",
-                          "--warmup", "3", "--workload", "small"], capture_output=True, text=True, timeout=600)
+                          "--warmup", "3", "--workload", "small", "--ref-threads", "1"],
+                         capture_output=True, text=True, timeout=600)
     assert out.returncode == 0, out.stderr
     lines = [l for l in out.stdout.splitlines() if l.strip()]
     assert len(lines) == 1
@@ -18,6 +19,17 @@ def test_reference_arm_prints_one_json_line():
     assert rec["value"] > 0 and rec["cpu_baseline"]["kind"] == "oracle" and rec["cpu_baseline"]["cores"] == 1
     assert rec["e2e"] == {"value": rec["value"], "unit": "params/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}
     assert rec["config"]["workload"].startswith("small_signum")
+
+
+def test_reference_arm_defaults_to_the_largest_configuration_on_all_cores():
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--steps", "1",
+                          "--warmup", "3", "--ref-sample", "400000"], capture_output=True, text=True, timeout=900)
+    assert out.returncode == 0, out.stderr
+    rec = json.loads(out.stdout.strip().splitlines()[-1])
+    assert rec["config"]["workload"] == "bertlarge_d335141888_M16" and rec["config"]["M"] == 16
+    cb = rec["cpu_baseline"]
+    assert cb["host_cores"] >= cb["cores"] >= 1 and cb["value"] == rec["value"] > 0
+    assert "disjoint 32-aligned slices" in cb["sample"]
 
 
 def test_other_ranks_of_the_reference_arm_do_nothing():

@@ -160,6 +160,92 @@ def test_whole_step_small(M):
                 assert_same_f32(f32(md).reshape(-1), m_ref, "m")
 
 
+# Odd vector lengths large enough that the launchers pick their largest tiles (16 and 32 elements per
+# thread), so that those instantiations meet a ragged last tile, a last word with pad bits, and rows
+# whose stride exceeds d.
+BIG_ODD_D = [5_000_003, (1 << 23) + 4099]
+
+
+def big_inputs(M, d, ld, seed, with_m=True):
+    r = np.random.default_rng(seed)
+    g = r.standard_normal((M, ld), dtype=np.float32)
+    g[:, ::97] = 0.0
+    g[:, 5::1013] *= np.float32(1e-3)
+    m = (0.3 * r.standard_normal((M, ld), dtype=np.float32)) if with_m else None
+    x = r.standard_normal(d + 8, dtype=np.float32)
+    x[d:] = CANARY_F
+    return g, m, x
+
+
+def check_rows(bits, ref, M, ldw, W, what):
+    got = u32(bits)
+    assert np.array_equal(got[:, :W], ref.reshape(M, ldw)[:, :W]), what
+    assert np.all(got[:, W:] == np.uint32(0xDEADBEEF)), what + ": row padding written"
+
+
+@pytest.mark.parametrize("d", BIG_ODD_D)
+@pytest.mark.parametrize("M", [1, 3])
+def test_sign_pack_large_odd_d(d, M):
+    ld, W = wl.round_up(d, 4) + 8, oracle.words(d)
+    ldw = wl.round_up(W, 4) + 4
+    g, _, _ = big_inputs(M, d, ld, seed=d % 1000 + M, with_m=False)
+    bits = torch.full((M, ldw), CANARY_WORD, dtype=torch.int32, device=DEV)
+    B.sign_pack(torch.from_numpy(g).to(DEV), M, d, ld, bits, ldw)
+    check_rows(bits, oracle.sign_pack(g.reshape(-1), M, d, ld=ld, ldw=ldw), M, ldw, W, "sign_pack d=%d M=%d" % (d, M))
+
+
+@pytest.mark.parametrize("d", BIG_ODD_D)
+@pytest.mark.parametrize("M,beta,with_m", [(1, 0.0, False), (8, 0.0, False), (16, 0.9, True), (5, 0.9, True)])
+def test_whole_step_large_odd_d(d, M, beta, with_m):
+    ld, W = wl.round_up(d, 4) + 8, oracle.words(d)
+    ldw = wl.round_up(W, 4) + 4
+    g, m, x = big_inputs(M, d, ld, seed=d % 1000 + 7 * M, with_m=with_m)
+    gd, xd = torch.from_numpy(g).to(DEV), torch.from_numpy(x).to(DEV)
+    md = torch.from_numpy(m).to(DEV) if with_m else None
+    bits = torch.full((M, ldw), CANARY_WORD, dtype=torch.int32, device=DEV)
+    vote = torch.full((W + 4,), CANARY_WORD, dtype=torch.int32, device=DEV)
+    B.signsgd_step(xd, gd, md, M, d, ld, beta, 1e-3, bits, ldw, vote)
+    x_ref = x[:d].copy()
+    m_ref = m.copy().reshape(-1) if with_m else None
+    b_ref, v_ref = oracle.signsgd_step(x_ref, g.reshape(-1), m_ref, M, d, beta, 1e-3, ld=ld, ldw=ldw)
+    check_rows(bits, b_ref, M, ldw, W, "bits d=%d M=%d" % (d, M))
+    assert np.array_equal(u32(vote)[:W], v_ref) and np.all(u32(vote)[W:] == np.uint32(0xDEADBEEF))
+    gx = f32(xd)
+    assert_same_f32(gx[:d], x_ref, "x")
+    assert np.all(gx[d:] == np.float32(CANARY_F))
+    if with_m:
+        gm = f32(md)
+        assert_same_f32(gm.reshape(-1), m_ref, "m")                 # includes the untouched elements >= d
+        assert np.array_equal(gm[:, d:].view(np.uint32), m[:, d:].view(np.uint32))
+
+
+@pytest.mark.parametrize("d", BIG_ODD_D)
+@pytest.mark.parametrize("M", [7, 16])
+def test_warmup_large_odd_d(d, M):
+    ld, W = wl.round_up(d, 4) + 8, oracle.words(d)
+    ldw = wl.round_up(W, 4) + 4
+    g, m, x = big_inputs(M, d, ld, seed=d % 1000 + 3 * M)
+    gd = torch.from_numpy(g).to(DEV)
+    md = torch.from_numpy(m).to(DEV)
+    bits = torch.full((M, ldw), CANARY_WORD, dtype=torch.int32, device=DEV)
+    B.signum_warmup_pack(gd, md, M, d, ld, 0.9, bits, ldw)
+    m_ref = m.copy().reshape(-1)
+    check_rows(bits, oracle.signum_warmup_pack(g.reshape(-1), m_ref, M, d, 0.9, ld=ld, ldw=ldw), M, ldw, W, "warm-up pack")
+    assert_same_f32(f32(md).reshape(-1), m_ref, "m after warm-up pack")
+    md, xd = torch.from_numpy(m).to(DEV), torch.from_numpy(x).to(DEV)
+    bits.fill_(CANARY_WORD)
+    vote = torch.full((W + 4,), CANARY_WORD, dtype=torch.int32, device=DEV)
+    B.signsgd_warmup_step(xd, gd, md, M, d, ld, 0.9, 1e-3, bits, ldw, vote)
+    m_ref, x_ref = m.copy().reshape(-1), x[:d].copy()
+    b_ref, v_ref = oracle.signsgd_warmup_step(x_ref, g.reshape(-1), m_ref, M, d, 0.9, 1e-3, ld=ld, ldw=ldw)
+    check_rows(bits, b_ref, M, ldw, W, "warm-up step bits")
+    assert np.array_equal(u32(vote)[:W], v_ref) and np.all(u32(vote)[W:] == np.uint32(0xDEADBEEF))
+    gx = f32(xd)
+    assert_same_f32(gx[:d], x_ref, "x")
+    assert np.all(gx[d:] == np.float32(CANARY_F))
+    assert_same_f32(f32(md).reshape(-1), m_ref, "m")
+
+
 def test_empty_input_launches_nothing():
     z = torch.zeros(4, dtype=torch.float32, device=DEV)
     b = torch.full((4,), CANARY_WORD, dtype=torch.int32, device=DEV)
@@ -492,11 +578,10 @@ def test_welford_and_density(d):
     phi_ref, l1, l2 = oracle.density(mean)
     phi = B.density(mean_d, d)
     assert abs(phi - phi_ref) <= 1e-11 * max(phi_ref, 1e-300)
-    sig = np.sqrt(m2.astype(np.float64)).astype(np.float32)      # sqrt in fp64, rounded once, as a stand-in
+    # the noise density phi(sigma) from the variances: the root form, against the oracle's
+    phi_s_ref, _, l2s = oracle.density_of_root(m2)
     phi_s = B.density(m2_d, d, root=True)
-    l1s = float(np.sqrt(m2.astype(np.float64)).sum())
-    l2s = float(m2.astype(np.float64).sum())
-    assert abs(phi_s - l1s * l1s / (d * l2s)) <= 1e-11 * phi_s if l2s > 0 else phi_s == 0.0
+    assert abs(phi_s - phi_s_ref) <= 1e-11 * phi_s_ref if l2s > 0 else phi_s == 0.0
 
 
 def test_density_of_dense_and_one_hot_vectors_gpu():
@@ -507,3 +592,6 @@ def test_density_of_dense_and_one_hot_vectors_gpu():
     one_hot[12345] = 4.0
     assert abs(B.density(one_hot, d) - 1.0 / d) < 1e-18
     assert B.density(torch.zeros(8, device=DEV), 8) == 0.0
+    # the same end points for a vector of variances through the root form
+    assert abs(B.density(torch.full((d,), 6.25, device=DEV), d, root=True) - 1.0) < 1e-12
+    assert abs(B.density(one_hot, d, root=True) - 1.0 / d) < 1e-18

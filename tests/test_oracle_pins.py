@@ -604,6 +604,30 @@ def test_density_of_dense_and_one_hot_vectors():
     assert abs(oracle.density(v)[0] - 0.25) < 1e-12
 
 
+def test_density_of_root_on_vectors_of_variances():
+    # Sec. 3's end points for the noise vector sigma, given as variances sigma^2:
+    # every component equally noisy -> 1; noise on one component only -> 1/d
+    d = 1000
+    assert abs(oracle.density_of_root(np.full(d, 6.25, dtype=np.float32))[0] - 1.0) < 1e-12
+    one = np.zeros(d, dtype=np.float32)
+    one[3] = 1e4                                    # e.g. the toy problem: noise on a single coordinate
+    assert abs(oracle.density_of_root(one)[0] - 1.0 / d) < 1e-15
+    assert oracle.density_of_root(np.zeros(4, dtype=np.float32))[0] == 0.0
+    v = np.zeros(d, dtype=np.float32)
+    v[:250] = 0.49
+    assert abs(oracle.density_of_root(v)[0] - 0.25) < 1e-9
+    # perfect squares: the roots are exact integers, so the sums are exact small integers
+    r = rng(84)
+    k = r.integers(0, 200, 5000)
+    sq = (k * k).astype(np.float32)
+    phi, l1, l2 = oracle.density_of_root(sq)
+    assert l1 == float(k.sum()) and l2 == float((k * k).sum())
+    assert phi == float(k.sum()) ** 2 / (5000 * float((k * k).sum()))
+    # half-normal scale mixture: sigma_i = |z_i| has phi -> 2/pi, from v = z^2
+    z = r.standard_normal(400_000)
+    assert abs(oracle.density_of_root((z * z).astype(np.float32))[0] - 2 / math.pi) < 5e-3
+
+
 def test_welford_matches_two_pass_mean_and_variance():
     r = rng(82)
     n, d = 40, 3000
