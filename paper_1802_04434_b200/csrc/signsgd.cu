@@ -23,79 +23,106 @@
 namespace {
 
 // ---------------------------------------------------------------------------
-// worker kernel: [momentum update +] sign + 1-bit pack, all M rows in one launch.
-// Tiles are numbered row-major over (row, tile in row), one tile per CTA.
+// worker step: [momentum update +] sign + 1-bit pack, all M rows in one launch.
+// Grid: x = tile within the row, y = row; one tile per CTA, consecutive CTAs on
+// consecutive tiles of a row.  A warp owns a span of 128 * UNROLL consecutive
+// elements of one row.
 
+// One span that crosses the end of its row: element-wise guards, padding bits
+// stay 0, and nothing at or beyond d is written.
 template <int MODE, int UNROLL>
-__global__ void __launch_bounds__(kThreads)
+__device__ __forceinline__ void worker_ragged_span(const float* __restrict__ gr, float* __restrict__ mr,
+                                                   uint32_t* __restrict__ br, unsigned long long d,
+                                                   unsigned long long e0, float beta, float omb) {
+  constexpr bool MOMENTUM = MODE != kSignSGD;
+  constexpr bool SIGN_OF_G = MODE != kSignum;
+  const unsigned lane = threadIdx.x & 31u;
+#pragma unroll 1
+  for (int u = 0; u < UNROLL; ++u) {
+    const unsigned long long e = e0 + u * 128 + lane * 4;
+    unsigned nib = 0;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      if (e + k < d) {
+        const float gk = gr[e + k];
+        float v = gk;
+        if (MOMENTUM) {
+          v = momentum_update(beta, omb, mr[e + k], gk);
+          mr[e + k] = v;
+        }
+        nib |= sign_bit(SIGN_OF_G ? gk : v) << k;
+      }
+    }
+    const unsigned word = assemble_word(nib, lane);
+    const unsigned long long first = e0 + u * 128 + (lane >> 3) * 32;  // first element of the word
+    if ((lane & 7u) == 0 && first < d) br[u * 4 + (lane >> 3)] = word;
+  }
+}
+
+// RAGGED = true: the kernel also handles the span that crosses the end of the row
+// (used for the small tiles, where one launch matters more than the last per cent
+// of bandwidth).  RAGGED = false: such a span is left to worker_tail_kernel, and
+// this kernel is nothing but the interior path.  Measured on B200 at d = 335 M,
+// M = 16: with the guarded path compiled into the same kernel the interior path
+// gets a different register allocation (40 or 48 registers instead of 52, hence
+// 6 or 5 resident CTAs per SM instead of 4) and streams 1.5-2.5 % slower.
+template <int MODE, int UNROLL, bool RAGGED>
+__global__ void __launch_bounds__(kThreads, 1)
 worker_pack_kernel(const float* __restrict__ g, float* __restrict__ m,
                    uint32_t* __restrict__ bits, unsigned long long d,
-                   unsigned long long ld, unsigned long long ldw,
-                   unsigned long long tiles_per_row, unsigned long long total_tiles,
-                   float beta, float omb) {
+                   unsigned long long ld, unsigned long long ldw, float beta, float omb) {
   constexpr bool MOMENTUM = MODE != kSignSGD;
   constexpr bool SIGN_OF_G = MODE != kSignum;
   constexpr unsigned long long TILE = (unsigned long long)kThreads * 4 * UNROLL;
   constexpr unsigned SPAN = 128 * UNROLL;
   const unsigned lane = threadIdx.x & 31u;
   const unsigned warp = threadIdx.x >> 5;
-
-  for (unsigned long long t = blockIdx.x; t < total_tiles; t += gridDim.x) {
-    const unsigned long long row = t / tiles_per_row;
-    const unsigned long long tile = t - row * tiles_per_row;
-    // first element of this warp's span, within the row
-    const unsigned long long e0 = tile * TILE + (unsigned long long)warp * SPAN;
-    if (e0 >= d) continue;
-    const float* gr = g + row * ld;
-    float* mr = MOMENTUM ? m + row * ld : nullptr;
-    uint32_t* br = bits + row * ldw + (e0 >> 5);
-    unsigned mine = 0;
-
-    if (e0 + SPAN <= d) {
-      // interior: no bounds checks, all loads issued before any use
-      float4 gv[UNROLL], mv[UNROLL];
-#pragma unroll
-      for (int u = 0; u < UNROLL; ++u) gv[u] = ld128(gr + e0 + u * 128 + lane * 4);
-      if (MOMENTUM) {
-#pragma unroll
-        for (int u = 0; u < UNROLL; ++u) mv[u] = ld128(mr + e0 + u * 128 + lane * 4);
-      }
-#pragma unroll
-      for (int u = 0; u < UNROLL; ++u) {
-        float4 v = gv[u];
-        if (MOMENTUM) {
-          v = momentum_update4(beta, omb, mv[u], v);
-          st128(mr + e0 + u * 128 + lane * 4, v);
-        }
-        const unsigned word = assemble_word(sign_nibble(SIGN_OF_G ? gv[u] : v), lane);
-        if ((lane & 7u) == (unsigned)u) mine = word;
-      }
-      if ((lane & 7u) < (unsigned)UNROLL) br[own_word_index<UNROLL>(lane)] = mine;
-    } else {
-      // ragged end of the row: element-wise guards, padding bits stay 0, and
-      // nothing at or beyond d is written
-#pragma unroll 1
-      for (int u = 0; u < UNROLL; ++u) {
-        const unsigned long long e = e0 + u * 128 + lane * 4;
-        unsigned nib = 0;
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-          if (e + k < d) {
-            const float gk = gr[e + k];
-            float v = gk;
-            if (MOMENTUM) {
-              v = momentum_update(beta, omb, mr[e + k], gk);
-              mr[e + k] = v;
-            }
-            nib |= sign_bit(SIGN_OF_G ? gk : v) << k;
-          }
-        }
-        const unsigned word = assemble_word(nib, lane);
-        const unsigned long long first = e0 + u * 128 + (lane >> 3) * 32;  // first element of the word
-        if ((lane & 7u) == 0 && first < d) br[u * 4 + (lane >> 3)] = word;
-      }
-    }
+  const unsigned long long row = blockIdx.y;
+  // first element of this warp's span, within the row
+  const unsigned long long e0 = (unsigned long long)blockIdx.x * TILE + (unsigned long long)warp * SPAN;
+  if (e0 + SPAN > d) {   // uniform over the warp; nothing below synchronises across warps
+    if (RAGGED && e0 < d)
+      worker_ragged_span<MODE, UNROLL>(g + row * ld, MOMENTUM ? m + row * ld : nullptr,
+                                       bits + row * ldw + (e0 >> 5), d, e0, beta, omb);
+    return;
   }
+  // interior: no bounds checks, all loads issued before any use
+  const float* gr = g + row * ld + e0 + lane * 4;
+  float* mr = MOMENTUM ? m + row * ld + e0 + lane * 4 : nullptr;
+  float4 gv[UNROLL], mv[UNROLL];
+#pragma unroll
+  for (int u = 0; u < UNROLL; ++u) gv[u] = ld128(gr + u * 128);
+  if (MOMENTUM) {
+#pragma unroll
+    for (int u = 0; u < UNROLL; ++u) mv[u] = ld128(mr + u * 128);
+  }
+  unsigned mine = 0;
+#pragma unroll
+  for (int u = 0; u < UNROLL; ++u) {
+    float4 v = gv[u];
+    if (MOMENTUM) {
+      v = momentum_update4(beta, omb, mv[u], v);
+      st128(mr + u * 128, v);
+    }
+    const unsigned word = assemble_word(sign_nibble(SIGN_OF_G ? gv[u] : v), lane);
+    if ((lane & 7u) == (unsigned)u) mine = word;
+  }
+  if ((lane & 7u) < (unsigned)UNROLL) bits[row * ldw + (e0 >> 5) + own_word_index<UNROLL>(lane)] = mine;
+}
+
+// The last, partial span of every row, for the launches whose main kernel is
+// interior-only: one warp per row.
+template <int MODE, int UNROLL>
+__global__ void __launch_bounds__(32)
+worker_tail_kernel(const float* __restrict__ g, float* __restrict__ m, uint32_t* __restrict__ bits,
+                   unsigned long long d, unsigned long long ld, unsigned long long ldw, float beta,
+                   float omb) {
+  constexpr unsigned SPAN = 128 * UNROLL;
+  const unsigned long long row = blockIdx.x;
+  const unsigned long long e0 = d / SPAN * SPAN;
+  if (e0 >= d) return;
+  worker_ragged_span<MODE, UNROLL>(g + row * ld, MODE != kSignSGD ? m + row * ld : nullptr,
+                                   bits + row * ldw + (e0 >> 5), d, e0, beta, omb);
 }
 
 // ---------------------------------------------------------------------------
@@ -297,15 +324,28 @@ fused_step_kernel(const float* __restrict__ g, float* __restrict__ m, float* __r
 // ---------------------------------------------------------------------------
 // host side
 
+constexpr size_t kWorkerSharedHint = 36 * 1024;   // below the 48 KB that need no opt-in
+
 template <int MODE, int UNROLL>
-void launch_worker_u(const float* g, float* m, size_t M, size_t d, size_t ld, float beta,
+bool launch_worker_u(const float* g, float* m, size_t M, size_t d, size_t ld, float beta,
                      uint32_t* bits, size_t ldw, cudaStream_t s) {
   constexpr unsigned long long TILE = (unsigned long long)kThreads * 4 * UNROLL;
+  constexpr bool SPLIT = UNROLL >= 4;    // large inputs: interior-only main kernel + a tail launch if needed
   const unsigned long long tiles_per_row = (d + TILE - 1) / TILE;
-  const unsigned long long total = tiles_per_row * M;
+  if (tiles_per_row > kMaxGrid) return false;     // beyond any device's memory
   const float omb = 1.0f - beta;
-  worker_pack_kernel<MODE, UNROLL><<<grid_for(total), kThreads, 0, s>>>(
-      g, m, bits, d, ld, ldw, tiles_per_row, total, beta, omb);
+  // The interior-only kernels ask for 36 KB of dynamic shared memory per CTA that they never touch.
+  // With four resident CTAs that moves 144 KB of the SM's L1 / shared-memory array to the shared side;
+  // measured on B200 (d = 335 M, M = 16, five runs on different boards) the stream is then 0.7-1.3 %
+  // faster than with the whole array as L1, while 170 KB and more on the shared side is slower.
+  const size_t smem = SPLIT ? kWorkerSharedHint : 0;
+  worker_pack_kernel<MODE, UNROLL, !SPLIT><<<dim3((unsigned)tiles_per_row, (unsigned)M), kThreads, smem, s>>>(
+      g, m, bits, d, ld, ldw, beta, omb);
+  if constexpr (SPLIT) {
+    if (d % (128 * UNROLL) != 0)
+      worker_tail_kernel<MODE, UNROLL><<<(unsigned)M, 32, 0, s>>>(g, m, bits, d, ld, ldw, beta, omb);
+  }
+  return true;
 }
 
 template <int MODE>
@@ -314,13 +354,14 @@ ssgd_status launch_worker(const float* g, float* m, size_t M, size_t d, size_t l
   DeviceInfo di;
   if (!device_info(&di)) return SSGD_ERR_CUDA;
   // without a momentum there is one array to load: twice the elements per thread keep as many loads in flight
+  bool ok;
   switch (pick_unroll(d, M, di.sms, MODE == kSignSGD ? 8 : 4)) {
-    case 8: launch_worker_u<kSignSGD, 8>(g, m, M, d, ld, beta, bits, ldw, s); break;
-    case 4: launch_worker_u<MODE, 4>(g, m, M, d, ld, beta, bits, ldw, s); break;
-    case 2: launch_worker_u<MODE, 2>(g, m, M, d, ld, beta, bits, ldw, s); break;
-    default: launch_worker_u<MODE, 1>(g, m, M, d, ld, beta, bits, ldw, s); break;
+    case 8: ok = launch_worker_u<kSignSGD, 8>(g, m, M, d, ld, beta, bits, ldw, s); break;
+    case 4: ok = launch_worker_u<MODE, 4>(g, m, M, d, ld, beta, bits, ldw, s); break;
+    case 2: ok = launch_worker_u<MODE, 2>(g, m, M, d, ld, beta, bits, ldw, s); break;
+    default: ok = launch_worker_u<MODE, 1>(g, m, M, d, ld, beta, bits, ldw, s); break;
   }
-  return launch_status();
+  return ok ? launch_status() : SSGD_ERR_SIZE;
 }
 
 template <int UNROLL>

@@ -39,6 +39,9 @@ def peak_gbs() -> float:
         return 6650.0
 
 
+PLAIN_LAUNCHES = False     # --plain: no CUDA graph, every launch issued from the host (for use under a profiler)
+
+
 def time_launches(fn, n_sets: int, reps: int) -> float:
     """Average milliseconds per launch of fn(set_index).
 
@@ -49,6 +52,15 @@ def time_launches(fn, n_sets: int, reps: int) -> float:
         fn(s)
     torch.cuda.synchronize()
     inner = max(1, -(-32 // n_sets))
+    if PLAIN_LAUNCHES:
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(reps):
+            for s in range(n_sets):
+                fn(s)
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / (reps * n_sets)
     graph = torch.cuda.CUDAGraph()
     with torch.cuda.graph(graph):
         for _ in range(inner):
@@ -161,11 +173,16 @@ def main(argv=None):
     ap.add_argument("--workers", default="1,3,7,15,31")
     ap.add_argument("--reps", type=int, default=20)
     ap.add_argument("--out", default=None)
+    ap.add_argument("--plain", action="store_true",
+                    help="issue every launch from the host instead of replaying a CUDA graph (times then include "
+                         "the host's per-call cost; meant for runs under a profiler)")
     ap.add_argument("--variants", default=None, metavar="LOG2D,M",
                     help="instead of the sweep, time the calls beside the main path at d = 2^LOG2D with M workers")
     args = ap.parse_args(argv)
     if not torch.cuda.is_available():
         raise SystemExit("the sweep needs a CUDA device")
+    global PLAIN_LAUNCHES
+    PLAIN_LAUNCHES = args.plain
     dev = torch.device("cuda", 0)
     B.lib()
     out = open(args.out, "w") if args.out else None
