@@ -42,8 +42,15 @@ FALLBACK_HBM_GBS = 6650.0
 # captures summarised in profiles/ (taken at a reduced d with the same M and kernels; the path is
 # elementwise, so traffic grows in proportion to d).  Valid only while the kernel sources are unchanged.
 NCU_TRAFFIC = {
-    "source_sha256": "",
-    "per_param": {},
+    "source_sha256": "e34279a2ea5ad974b5fa153003426cffda3bae16ec103dc6dbac7cf31ccc96a4",
+    "per_param": {
+        # profiles/worker_vote_apply_kernels_d2p25_M16_ncu_full.md
+        "worker_pack_kernel:M16": {"bytes_per_param": (4.295064e9 + 2.164399e9) / 33554432, "d": 33554432},
+        "vote_kernel:M16": {"bytes_per_param": (67.118e6 + 0.771e6) / 33554432, "d": 33554432},
+        # (apply_kernel: in the reduced capture x is partly L2-resident, so its traffic does not scale with d)
+        # profiles/fused_step_kernel_resnet50_M7_ncu_full.md (captured at full size)
+        "fused_step_kernel:M7": {"bytes_per_param": (1.533690e9 + 793.246464e6) / 25557056, "d": 25557056},
+    },
 }
 
 KERNEL_SOURCES = ("signsgd.cu", "device_common.cuh", "host_common.h")
