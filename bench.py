@@ -42,7 +42,7 @@ FALLBACK_HBM_GBS = 6650.0
 # captures summarised in profiles/ (taken at a reduced d with the same M and kernels; the path is
 # elementwise, so traffic grows in proportion to d).  Valid only while the kernel sources are unchanged.
 NCU_TRAFFIC = {
-    "source_sha256": "e34279a2ea5ad974b5fa153003426cffda3bae16ec103dc6dbac7cf31ccc96a4",
+    "source_sha256": "14fc0fb97f57511dbb3fe65a3c20fe277d739ec90ed0f5372787283f4173ece0",
     "per_param": {
         # profiles/worker_vote_apply_kernels_d2p25_M16_ncu_full.md
         "worker_pack_kernel:M16": {"bytes_per_param": (4.295064e9 + 2.164399e9) / 33554432, "d": 33554432},
@@ -57,12 +57,18 @@ KERNEL_SOURCES = ("signsgd.cu", "device_common.cuh", "host_common.h")
 
 
 def kernel_source_digest():
+    """sha256 of the kernel sources with comments and white space removed: an edit of a comment does not
+    invalidate the ncu figures, an edit of the code does."""
     import hashlib
+    import re
     h = hashlib.sha256()
     try:
         for name in KERNEL_SOURCES:
-            with open(os.path.join(ROOT, "paper_1802_04434_b200", "csrc", name), "rb") as fh:
-                h.update(fh.read())
+            with open(os.path.join(ROOT, "paper_1802_04434_b200", "csrc", name), "r") as fh:
+                text = fh.read()
+            text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+            text = re.sub(r"//[^\n]*", "", text)
+            h.update("".join(text.split()).encode())
     except OSError:
         return None
     return h.hexdigest()
@@ -589,27 +595,43 @@ def run_workers(args, torch, B, multi, dev, rank, local_rank, world):
     ws = multi.WorkerStep(d, dev)
     stream = torch.cuda.current_stream()
     K, Wm = args.steps, args.warmup
+    small = 2 * ld * 4 <= (256 << 20)       # one rank's g + m would stay in L2 from step to step
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev) if small else None
     step = lambda ev=None: ws.step(x, g, m, cfg.beta, cfg.delta, events=ev)
     for _ in range(Wm):
         step()
+
+    def block():
+        """K steps, each with its four events; returns a reader of (step, pack, exchange, vote + apply) ms sums."""
+        marks = []
+        for _ in range(K):
+            ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+            step(ev)
+            if flush is not None:
+                flush.zero_()
+            marks.append(ev)
+        return lambda: [sum(e[i].elapsed_time(e[j]) for e in marks) for i, j in ((0, 3), (0, 1), (1, 2), (2, 3))]
+
     sampler = ClockSampler(local_rank)
     multi.barrier(dev)
     sampler.start()
-    marks = []
     t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     t0.record(stream)
-    for _ in range(K):
-        ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
-        step(ev)
-        marks.append(ev)
+    read = block()
     t1.record(stream)
     multi.barrier(dev)
-    sampler.stop()
-    elapsed_ms = t0.elapsed_time(t1)
-    pack_ms = sum(e[0].elapsed_time(e[1]) for e in marks) / K
-    xchg_ms = sum(e[1].elapsed_time(e[2]) for e in marks) / K
-    rest_ms = sum(e[2].elapsed_time(e[3]) for e in marks) / K
+    step_sum, pack_sum, xchg_sum, rest_sum = read()
+    # without a flush the K steps are timed as one region; with it, as the sum of the per-step event pairs
+    elapsed_ms = step_sum if flush is not None else t0.elapsed_time(t1)
+    pack_ms, xchg_ms, rest_ms = pack_sum / K, xchg_sum / K, rest_sum / K
     elapsed_ms, pack_ms, xchg_ms, rest_ms = multi.max_over_ranks([elapsed_ms, pack_ms, xchg_ms, rest_ms], dev)
+    # Clock samples must be of timed work: a short region is repeated under the sampler.  Every block holds
+    # collectives, so all ranks must run the same number of them: it is derived from the reduced time.
+    extra = min(2000, max(0, int(150.0 / max(elapsed_ms, 1e-3))))
+    for _ in range(extra):
+        block()
+    multi.barrier(dev)
+    sampler.stop()
     same = multi.all_ranks_equal(ws.vote)
     if rank == 0:
         peak, peak_kind = measured_peak()
@@ -619,7 +641,9 @@ def run_workers(args, torch, B, multi, dev, rank, local_rank, world):
             "metric": METRIC, "value": d * K / (elapsed_ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K,
             "warmup": Wm, "ms_per_step": elapsed_ms / K, "higher_is_better": True, "scaling": "strong",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": workload_config(cfg, world, "workers"),
+            "config": dict(workload_config(cfg, world, "workers"),
+                           l2="L2 flushed between timed steps by writing a 256 MiB buffer; step time = sum of per-step "
+                              "event pairs" if small else "g + m per step exceed L2 (no flush needed)"),
             "wire_bits_per_step_table1": 2 * Mw * d,
             "wire_bytes_sent_per_rank_per_step": ws.ldw * 4 * (world - 1),
             "exchange": {"collective": "all_gather_into_tensor of ceil(d/32)-word rows (NCCL)", "ms": xchg_ms,
@@ -637,7 +661,8 @@ def run_workers(args, torch, B, multi, dev, rank, local_rank, world):
                          "unit": "GB/s", "frac": pack_bytes / (pack_ms * 1e-3) / 1e9 / peak, "traffic": None},
             "votes_identical_on_all_ranks": bool(same),
             "gpu_launches": 3 * K,
-            "clocks": sampler.summary(),
+            "clocks": sampler.summary("the %d-step block was repeated %d more times inside the sampling window"
+                                      % (K, extra) if extra else None),
         }
         print(json.dumps(line), flush=True)
     multi.finish()

@@ -67,9 +67,9 @@ constexpr int kThreads = 256;
 // What a worker sends, and whether it keeps a momentum:
 //   kSignSGD       bit = sign(g)                       (Algorithm 1 / Algorithm 3 as printed)
 //   kSignum        m <- beta m + (1-beta) g, bit = sign(m)            (Algorithm 2)
-//   kSignumWarmup  m updated as in kSignum, bit = sign(g): the first C(beta)
-//                  iterations of Theorem 3, which accumulate the momentum as
-//                  normal but step with the sign of the stochastic gradient
+//   kSignumWarmup  m updated as in kSignum, bit = sign(g): the warm-up iterations
+//                  of Theorem 3 (the first C(beta) ones), whose momentum is
+//                  already the running average while the vote is still on g
 constexpr int kSignSGD = 0;
 constexpr int kSignum = 1;
 constexpr int kSignumWarmup = 2;

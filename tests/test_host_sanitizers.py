@@ -51,3 +51,27 @@ def test_the_sanitizer_run_does_catch_a_planted_overrun(tmp_path):
     assert res.returncode == 0, res.stderr
     run = subprocess.run([exe], capture_output=True, text=True, timeout=600)
     assert run.returncode != 0 and "AddressSanitizer" in run.stderr
+
+
+@pytest.mark.skipif(shutil.which("nvcc") is None and not os.path.exists("/usr/local/cuda/bin/nvcc"), reason="needs nvcc")
+def test_host_argument_checks_are_clean_under_asan_and_ubsan(tmp_path):
+    """The CUDA library's host layer (argument checks, size arithmetic, the warm-up length scan) built with the
+    host sanitizers and driven through every entry point's rejection and empty-input paths; runs without a GPU
+    because none of these calls may reach a launch."""
+    nvcc = shutil.which("nvcc") or "/usr/local/cuda/bin/nvcc"
+    csrc = os.path.join(ROOT, "paper_1802_04434_b200", "csrc")
+    exe = str(tmp_path / "abi_sanitized")
+    cmd = [nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-O1", "-std=c++17", "--fmad=false",
+           "-I", os.path.join(ROOT, "include"),
+           "-Xcompiler", "-fsanitize=address", "-Xcompiler", "-fsanitize=undefined",
+           "-Xcompiler", "-fno-sanitize-recover=all",
+           *[os.path.join(csrc, n) for n in ("signsgd.cu", "variants.cu", "stats.cu")],
+           os.path.join(ROOT, "tests", "sanitizer_abi_driver.cpp"), "-o", exe]
+    res = subprocess.run(cmd, capture_output=True, text=True, timeout=900)
+    assert res.returncode == 0, res.stderr[-2000:]
+    # the CUDA runtime reserves address ranges that ASan's shadow-gap protection would refuse
+    env = dict(os.environ, ASAN_OPTIONS="protect_shadow_gap=0:detect_leaks=0", UBSAN_OPTIONS="print_stacktrace=1")
+    run = subprocess.run([exe], capture_output=True, text=True, timeout=300, env=env)
+    assert run.returncode == 0, run.stdout + run.stderr[-2000:]
+    assert "all checks passed" in run.stdout
+    assert "runtime error" not in run.stderr and "AddressSanitizer" not in run.stderr
