@@ -316,8 +316,8 @@ def run_reference(args):
 
 def workload_config(cfg, n_gpus, mode="shards"):
     if mode == "workers":
-        par = ("Algorithm 3 with one worker per GPU: M = %d ranks, each packs its own sign row, all-gather of the "
-               "rows, local vote and apply" % n_gpus)
+        par = ("Algorithm 3 with one worker per GPU: M = %d ranks, each packs its own sign row, every row reaches "
+               "every rank, local vote and apply" % n_gpus)
     else:
         par = "independent shard of d per GPU, no collective" if n_gpus > 1 else "single GPU"
     return {"workload": cfg.name, "d": cfg.d, "M": cfg.M if mode != "workers" else n_gpus, "beta": cfg.beta,
@@ -592,7 +592,7 @@ def run_workers(args, torch, B, multi, dev, rank, local_rank, world):
     g = one.g(0, dev, shared)
     m = one.m0(dev) if momentum else None
     del shared
-    ws = multi.WorkerStep(d, dev)
+    ws = multi.WorkerStep(d, dev, exchange=args.exchange)
     stream = torch.cuda.current_stream()
     K, Wm = args.steps, args.warmup
     small = 2 * ld * 4 <= (256 << 20)       # one rank's g + m would stay in L2 from step to step
@@ -646,18 +646,20 @@ def run_workers(args, torch, B, multi, dev, rank, local_rank, world):
                               "event pairs" if small else "g + m per step exceed L2 (no flush needed)"),
             "wire_bits_per_step_table1": 2 * Mw * d,
             "wire_bytes_sent_per_rank_per_step": ws.ldw * 4 * (world - 1),
-            "exchange": {"collective": "all_gather_into_tensor of ceil(d/32)-word rows (NCCL)", "ms": xchg_ms,
+            "exchange": {"transport": "all_gather_into_tensor of ceil(d/32)-word rows (NCCL)" if args.exchange == "allgather"
+                         else "peer stores from the worker kernel (symmetric memory) + one barrier", "ms": xchg_ms,
                          "share_of_step": xchg_ms / (elapsed_ms / K)},
             "kernels": [
-                {"kernel": "worker_pack_kernel", "ms_per_launch": pack_ms, "bytes_per_launch": pack_bytes,
+                {"kernel": "worker_pack_kernel" if args.exchange == "allgather" else "pack_scatter_kernel",
+                 "ms_per_launch": pack_ms, "bytes_per_launch": pack_bytes,
                  "achieved_gbs": pack_bytes / (pack_ms * 1e-3) / 1e9,
                  "frac": pack_bytes / (pack_ms * 1e-3) / 1e9 / peak},
                 {"kernel": "vote_kernel + apply_kernel", "ms_per_launch": rest_ms,
                  "bytes_per_launch": (vote_bpp(Mw) + APPLY_BPP) * d,
                  "achieved_gbs": (vote_bpp(Mw) + APPLY_BPP) * d / (rest_ms * 1e-3) / 1e9,
                  "frac": (vote_bpp(Mw) + APPLY_BPP) * d / (rest_ms * 1e-3) / 1e9 / peak}],
-            "roofline": {"kernel": "worker_pack_kernel", "bound": "hbm",
-                         "achieved": pack_bytes / (pack_ms * 1e-3) / 1e9, "peak": peak, "peak_kind": "of " + peak_kind,
+            "roofline": {"kernel": "worker_pack_kernel" if args.exchange == "allgather" else "pack_scatter_kernel",
+                         "bound": "hbm", "achieved": pack_bytes / (pack_ms * 1e-3) / 1e9, "peak": peak, "peak_kind": "of " + peak_kind,
                          "unit": "GB/s", "frac": pack_bytes / (pack_ms * 1e-3) / 1e9 / peak, "traffic": None},
             "votes_identical_on_all_ranks": bool(same),
             "gpu_launches": 3 * K,
@@ -679,6 +681,8 @@ def main():
     ap.add_argument("--mode", choices=["shards", "workers"], default="shards",
                     help="shards: every GPU simulates all M workers on its own shard of parameters (no collective); "
                          "workers: one worker per GPU, sign rows all-gathered (Algorithm 3 as a distributed step)")
+    ap.add_argument("--exchange", choices=["allgather", "p2p"], default="allgather",
+                    help="--mode workers: how the sign rows travel (a collective, or peer stores from the worker kernel)")
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--e2e-warmup", type=int, default=1)

@@ -227,6 +227,37 @@ ssgd_status ssgd_signsgd_step_host(float* x, const float* g_host, float* m,
                                    uint32_t* vote_ws, uint32_t* vote_host,
                                    void* stream);
 
+/* Most ranks one ssgd_signum_momentum_pack_scatter call can send to. */
+#define SSGD_MAX_PEERS 64
+
+/* Algorithm 3 with one worker per GPU, the worker's half of a step in one kernel:
+ * Algorithm 2's momentum update on THIS worker's g and m and the 1-bit packing of
+ * its sign (exactly ssgd_signum_momentum_pack with M = 1; m == NULL with beta == 0
+ * sends sign(g) as Algorithm 3 prints it), fused with the transport of Algorithm
+ * 3's "pull sign(g_m)": every packed word is stored directly into row `row` of the
+ * rows buffer of each of P ranks, so that afterwards every rank holds this
+ * worker's d bits (Table 1: d bits up per worker) without a separate collective.
+ *   g      in      DEVICE [d] (16-byte aligned), this worker's gradient
+ *   m      in/out  DEVICE [d], updated in place; NULL allowed iff beta == 0
+ *   rows   in      HOST array of P DEVICE pointers (read during the call only):
+ *                  rows[r] is the [.][ldw] rows buffer of rank r, 16-byte aligned;
+ *                  it may live in another GPU's memory that this GPU can write
+ *                  (peer access enabled / symmetric memory), or in this GPU's own.
+ *                  1 <= P <= SSGD_MAX_PEERS; list this rank's own buffer too.
+ *   row            this worker's index: words go to rows[r] + row * ldw + j,
+ *                  j < W; words W..ldw-1 of the row are not written; bits >= d are 0.
+ *   ldw            row stride in words, a multiple of 4, >= W.
+ * The kernel only WRITES the destination rows (plain 32-bit stores) and contains
+ * no waits.  Ordering between ranks is the caller's: before a rank votes on its
+ * rows buffer, every rank's call must have completed (e.g. a barrier across the
+ * ranks enqueued after this call); before a rows buffer is written again, its
+ * owner must have finished reading it.  Errors as for ssgd_signum_momentum_pack;
+ * a NULL entry of rows gives SSGD_ERR_NULL, P or row out of range SSGD_ERR_SIZE. */
+ssgd_status ssgd_signum_momentum_pack_scatter(const float* g, float* m, size_t d,
+                                              float beta, uint32_t* const* rows,
+                                              size_t P, size_t row, size_t ldw,
+                                              void* stream);
+
 /* Capacity, in 32-bit words, of the scratch area that ssgd_signsgd_step_noalloc
  * uses (16 MiB of device memory per GPU that loads the library, held until the
  * process exits). */

@@ -67,6 +67,7 @@ def lib() -> ctypes.CDLL:
         "ssgd_density_sums": [vp, sz, ci, vp, vp],
         "ssgd_signsgd_step_host": [vp, vp, vp, sz, sz, sz, f32, f32, vp, vp, sz, vp, vp, vp],
         "ssgd_signsgd_step_noalloc": [vp, vp, vp, sz, sz, sz, f32, f32, vp],
+        "ssgd_signum_momentum_pack_scatter": [vp, vp, sz, f32, vp, sz, sz, sz, vp],
     }
     for name, args in sigs.items():
         fn = getattr(L, name)
@@ -285,6 +286,30 @@ def signsgd_step_host(x: torch.Tensor, g_host: torch.Tensor, m: Optional[torch.T
         _ptr(g_stage, torch.float32, "g_stage"), _ptr(bits_ws, WORD_DTYPE, "bits_ws"), ldw,
         _ptr(vote_ws, WORD_DTYPE, "vote_ws"), _ptr(vote_host, WORD_DTYPE, "vote_host", cuda=False),
         _stream(stream)), "ssgd_signsgd_step_host")
+
+
+MAX_PEERS = 64
+
+
+def signum_momentum_pack_scatter(g: torch.Tensor, m: Optional[torch.Tensor], d: int, beta: float, rows, row: int,
+                                 ldw: int, stream=None) -> None:
+    """One worker's momentum update + sign packing, with its words stored into row `row` of every rank's
+    rows buffer.  `rows` is a sequence with one entry per rank: a device tensor of int32 words (this
+    GPU's own memory) or a raw device address as int (another GPU's memory this GPU can write)."""
+    _need(g, d, "g")
+    if m is not None:
+        _need(m, d, "m")
+    addrs = []
+    for i, r in enumerate(rows):
+        if isinstance(r, torch.Tensor):
+            _need(r, (row + 1) * ldw, "rows[%d]" % i)
+            addrs.append(_ptr(r, WORD_DTYPE, "rows[%d]" % i))
+        else:
+            addrs.append(int(r))
+    table = (ctypes.c_void_p * len(addrs))(*addrs)
+    _check(lib().ssgd_signum_momentum_pack_scatter(
+        _ptr(g, torch.float32, "g"), _ptr(m, torch.float32, "m"), d, beta, table, len(addrs), row, ldw,
+        _stream(stream)), "ssgd_signum_momentum_pack_scatter")
 
 
 NOALLOC_SCRATCH_WORDS = 4 << 20

@@ -7,7 +7,8 @@ Two ways to use several GPUs:
   workers) and runs the same kernels on it.  The only communication is a barrier around the timed
   region and a max-reduction of the per-rank device times.
 * workers (`WorkerStep`): Algorithm 3 as the paper states it, one worker per rank, with one exchange
-  per step: an all-gather of the packed sign rows.
+  per step: an all-gather of the packed sign rows, either as a collective or done by the worker kernel
+  itself through peer stores.
 
 Both go through ``torch.distributed`` (NCCL on GPUs, gloo in the CPU tests).
 """
@@ -83,26 +84,39 @@ class WorkerStep:
     Rank r keeps its own gradient g_r, its own momentum m_r and a replica of x.  One step is
       1. worker block: m_r <- beta m_r + (1 - beta) g_r and the 1-bit sign row of it (or of g_r when
          there is no momentum), one launch on this rank's data (M = 1);
-      2. the exchange, in place of Algorithm 3's "pull sign(g_m)": an all-gather of the W-word rows, d bits
-         up per worker as in Table 1; rank r's row lands in row r of a local [world][ldw] buffer in
-         this GPU's own memory;
+      2. the exchange, in place of Algorithm 3's "pull sign(g_m)": every rank's W-word row reaches every
+         rank, d bits up per worker as in Table 1; rank r's row lands in row r of a [world][ldw] buffer
+         in each GPU's own memory;
       3. server block, done by every rank on its local copy of the M rows: the majority vote;
       4. worker block: x <- x - delta sign(vote) on the replica.  All ranks hold the same rows, so they
          compute the same vote and their replicas of x stay identical: no message "down" is needed.
 
-    The kernels only ever read local memory (the gathered rows), with plain loads.  `ops` supplies the
-    four compute calls (default: the CUDA binding); the CPU tests pass their own implementation.
+    Two transports for step 2:
+      exchange="allgather"  the rows are gathered by `all_gather_into_tensor` (NCCL on GPUs, gloo on CPU);
+      exchange="p2p"        steps 1 and 2 are ONE kernel (`signum_momentum_pack_scatter`): the lane that
+                            owns a sign word stores it into row r of every rank's rows buffer through
+                            peer pointers (torch symmetric memory), so the transfer overlaps the kernel's
+                            own g / m stream; a barrier across the ranks follows.  The rows buffers are
+                            double-buffered by step parity, so that a fast rank's next scatter cannot
+                            overwrite rows a slow rank is still voting on, with one barrier per step.
+    Either way the vote kernel only reads this GPU's own memory, with plain loads.  `ops` supplies the
+    compute calls (default: the CUDA binding); the CPU tests pass their own implementation.
     """
 
-    def __init__(self, d: int, device: torch.device, ops=None, group=None, world=None, rank=None):
+    def __init__(self, d: int, device: torch.device, ops=None, group=None, world=None, rank=None,
+                 exchange: str = "allgather"):
         if ops is None:
             from . import binding as ops   # the CUDA library; raises if it is missing
+        if exchange not in ("allgather", "p2p"):
+            raise ValueError("exchange must be 'allgather' or 'p2p'")
         self.ops = ops
         self.d = int(d)
         self.device = torch.device(device)
         self.group = group
+        self.exchange_kind = exchange
         # world / rank default to the process group's; a caller that moves the rows itself (several
         # workers emulated in one process) states them
+        in_group = dist.is_initialized() and world is None
         if world is None:
             world = dist.get_world_size(group) if dist.is_initialized() else 1
         if rank is None:
@@ -111,23 +125,64 @@ class WorkerStep:
         self.ld = round_up(self.d, 4)
         self.words = (self.d + 31) // 32
         self.ldw = round_up(self.words, 4)             # rows stay 16-byte aligned; at most 3 pad words
-        self.row = torch.zeros(self.ldw, dtype=torch.int32, device=self.device)
-        self.bits = torch.zeros(self.world, self.ldw, dtype=torch.int32, device=self.device)
         self.vote = torch.zeros(self.words, dtype=torch.int32, device=self.device)
+        self.sync = lambda: None
+        if exchange == "allgather":
+            self.row = torch.zeros(self.ldw, dtype=torch.int32, device=self.device)
+            self.bits = torch.zeros(self.world, self.ldw, dtype=torch.int32, device=self.device)
+        else:
+            self.parity = 0
+            if in_group and self.device.type == "cuda":
+                self._rendezvous()
+            elif in_group and self.world > 1:
+                raise ValueError("exchange='p2p' between processes needs CUDA devices (symmetric memory)")
+            else:
+                # no group: the rows buffers are ordinary local memory, and `connect` may point several
+                # emulated ranks of one process at one another
+                self.rows_buf = torch.zeros(2, self.world, self.ldw, dtype=torch.int32, device=self.device)
+                self.peer_rows = [[self.rows_buf[k]] for k in (0, 1)] if self.world == 1 else None
+            self.bits = self.rows_buf[0]
+
+    def _rendezvous(self) -> None:
+        """Rows buffers in symmetric memory: every rank learns every rank's buffer address."""
+        import torch.distributed._symmetric_memory as symm_mem
+        group = self.group if self.group is not None else dist.group.WORLD
+        self.rows_buf = symm_mem.empty((2, self.world, self.ldw), dtype=torch.int32, device=self.device)
+        self.rows_buf.zero_()
+        self.handle = symm_mem.rendezvous(self.rows_buf, group)
+        half = self.world * self.ldw * 4
+        self.peer_rows = [[int(self.handle.buffer_ptrs[r]) + k * half for r in range(self.world)] for k in (0, 1)]
+        self.sync = lambda: self.handle.barrier(channel=0)
+        self.sync()                                    # every rank's zeroing is done before any scatter
+
+    @staticmethod
+    def connect(ranks) -> None:
+        """Point the emulated ranks of ONE process (exchange="p2p", no process group) at one another."""
+        for ws in ranks:
+            ws.peer_rows = [[other.rows_buf[k] for other in ranks] for k in (0, 1)]
 
     def wire_bytes_sent_per_step(self) -> int:
         """Bytes this rank's row occupies on the wire, once per peer."""
         return self.ldw * 4 * (self.world - 1)
 
     def pack(self, g: torch.Tensor, m, beta: float) -> None:
-        """Worker block, first half: this worker's momentum update and its 1-bit sign row."""
-        if m is None:
+        """Worker block, first half: this worker's momentum update and its 1-bit sign row.  With the p2p
+        transport the same kernel also delivers the row to every rank."""
+        if self.exchange_kind == "p2p":
+            self.ops.signum_momentum_pack_scatter(g, m, self.d, beta if m is not None else 0.0,
+                                                  self.peer_rows[self.parity], self.rank, self.ldw)
+        elif m is None:
             self.ops.sign_pack(g, 1, self.d, self.ld, self.row, self.ldw)
         else:
             self.ops.signum_momentum_pack(g, m, 1, self.d, self.ld, beta, self.row, self.ldw)
 
     def exchange(self) -> None:
-        """Gather every rank's row into the local [world][ldw] buffer (row r <- rank r)."""
+        """After this, row r of the local [world][ldw] buffer holds rank r's words, on every rank."""
+        if self.exchange_kind == "p2p":
+            self.sync()                                # all ranks' scatter kernels have completed
+            self.bits = self.rows_buf[self.parity]
+            self.parity ^= 1
+            return
         if not dist.is_initialized() or dist.get_world_size(self.group) == 1:
             self.bits[self.rank].copy_(self.row)
             return

@@ -35,3 +35,16 @@ def majority_vote(bits, M, d, ldw, vote, stream=None):
 
 def sign_apply(x, vote, d, delta, stream=None):
     oracle.sign_apply(x.numpy(), _u32(vote), d, delta)
+
+
+def signum_momentum_pack_scatter(g, m, d, beta, rows, row, ldw, stream=None):
+    """One worker's row computed by the oracle and copied into row `row` of every rows buffer given."""
+    W = oracle.words(d)
+    gf = g.numpy().reshape(-1)[:d]
+    if m is None:
+        words = oracle.sign_pack(np.ascontiguousarray(gf), 1, d)
+    else:
+        mf = m.numpy().reshape(-1)[:d]                   # a view: updated in place
+        words = oracle.signum_momentum_pack(np.ascontiguousarray(gf), mf, 1, d, beta)
+    for r in rows:
+        _u32(r).reshape(-1)[row * ldw:row * ldw + W] = words[:W]

@@ -117,18 +117,15 @@ def test_single_process_worker_step_needs_no_group():
     assert np.array_equal(ws.vote.numpy().view(np.uint32), ref[-1][1])     # M = 1: the vote is the row
 
 
-@pytest.mark.gpu
-@pytest.mark.parametrize("world,d,momentum", [(2, 100_003, True), (8, 1_000_003, True), (8, 70_001, False),
-                                             (3, 4_200_000, True)])
-def test_emulated_ranks_on_one_gpu_match_the_oracle(world, d, momentum):
-    """Every emulated rank owns its buffers on cuda:0; the rows travel by plain device copies (the
-    stand-in for the all-gather), so each rank's vote kernel reads only its own gathered copy."""
-    from paper_1802_04434_b200 import binding as B
-    B.lib()
-    dev = torch.device("cuda", 0)
-    steps, beta, delta = 2, (0.9 if momentum else 0.0), 1e-3
+def run_emulated_ranks(world, d, momentum, exchange, dev, ops=None, steps=2):
+    """All ranks live in this process and run phase by phase, one after another (no kernel waits on another):
+    pack on every rank, then the exchange, then vote + apply on every rank.  Returns nothing; asserts parity
+    with the single-process oracle step over the stacked gradients."""
+    beta, delta = (0.9 if momentum else 0.0), 1e-3
     x0, g, m0 = worker_inputs(world, d, steps, seed=world * 31 + d, momentum=momentum)
-    ranks = [multi.WorkerStep(d, dev, world=world, rank=r) for r in range(world)]
+    ranks = [multi.WorkerStep(d, dev, ops=ops, world=world, rank=r, exchange=exchange) for r in range(world)]
+    if exchange == "p2p":
+        multi.WorkerStep.connect(ranks)                       # every rank's scatter writes into every rank's buffer
     xs = [torch.from_numpy(x0.copy()).to(dev) for _ in range(world)]
     ms = [torch.from_numpy(m0[r:r + 1].copy()).to(dev) if momentum else None for r in range(world)]
     ref, x_ref, m_ref = reference_run(x0, g, m0, d, beta, delta, momentum)
@@ -137,15 +134,21 @@ def test_emulated_ranks_on_one_gpu_match_the_oracle(world, d, momentum):
         gk = [torch.from_numpy(g[k, r:r + 1].copy()).to(dev) for r in range(world)]
         for r, ws in enumerate(ranks):
             ws.pack(gk[r], ms[r], beta)
-        for ws in ranks:                                       # the exchange: row r of everyone <- rank r's row
-            for r, src in enumerate(ranks):
-                ws.bits[r].copy_(src.row)
+        if exchange == "p2p":
+            for ws in ranks:
+                ws.exchange()                                   # parity flip; the words are already there
+        else:
+            for ws in ranks:                                    # stand-in for the all-gather: plain copies
+                for r, src in enumerate(ranks):
+                    ws.bits[r].copy_(src.row)
         for r, ws in enumerate(ranks):
             ws.vote_apply(xs[r], delta)
-        torch.cuda.synchronize()
+        if dev.type == "cuda":
+            torch.cuda.synchronize()
         for r, ws in enumerate(ranks):
             got = ws.bits.cpu().numpy().view(np.uint32)
-            assert np.array_equal(got[:, :W], ref[k][0][:, :W]) and np.all(got[:, W:] == 0)
+            assert np.array_equal(got[:, :W], ref[k][0][:, :W]), "step %d rank %d" % (k, r)
+            assert np.all(got[:, W:] == 0)
             assert np.array_equal(ws.vote.cpu().numpy().view(np.uint32), ref[k][1])
     ld = multi.round_up(d, 4)
     for r in range(world):
@@ -153,3 +156,117 @@ def test_emulated_ranks_on_one_gpu_match_the_oracle(world, d, momentum):
         if momentum:
             assert np.array_equal(ms[r].cpu().numpy().reshape(-1).view(np.uint32),
                                   m_ref[r * ld:(r + 1) * ld].view(np.uint32))
+
+
+@pytest.mark.parametrize("exchange", ["allgather", "p2p"])
+def test_emulated_ranks_host_logic_on_cpu(exchange):
+    # double-buffered rows, row placement and parity flips of the p2p transport; three steps so that a
+    # buffer is reused
+    import oracle_ops
+    run_emulated_ranks(3, 1000, True, exchange, torch.device("cpu"), ops=oracle_ops, steps=3)
+    run_emulated_ranks(2, 4099, False, exchange, torch.device("cpu"), ops=oracle_ops, steps=3)
+
+
+def test_unknown_exchange_is_refused():
+    with pytest.raises(ValueError):
+        multi.WorkerStep(100, torch.device("cpu"), exchange="nonsense")
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("world,d,momentum", [(2, 100_003, True), (8, 1_000_003, True), (5, 70_001, False),
+                                             (3, 5_000_003, True)])
+def test_emulated_ranks_with_the_fused_pack_and_scatter_kernel(world, d, momentum):
+    """The worker kernel that stores its words into every rank's rows buffer itself; here all buffers are on
+    cuda:0, so the peer pointers are ordinary device pointers."""
+    from paper_1802_04434_b200 import binding as B
+    B.lib()
+    run_emulated_ranks(world, d, momentum, "p2p", torch.device("cuda", 0), steps=3)
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("d", [1, 33, 4097, 100_003, 5_000_003])
+def test_pack_scatter_kernel_matches_oracle_and_touches_nothing_else(d):
+    from paper_1802_04434_b200 import binding as B
+    dev = torch.device("cuda", 0)
+    r = np.random.default_rng(d)
+    W = oracle.words(d)
+    ldw = multi.round_up(W, 4) + 4
+    P, rows_n, row = 3, 4, 2
+    g = r.standard_normal(d + 5).astype(np.float32)
+    g[::53] = 0.0
+    m = (0.2 * r.standard_normal(d + 5)).astype(np.float32)
+    for with_m, beta in ((True, 0.9), (False, 0.0)):
+        bufs = [torch.full((rows_n, ldw), -559038737, dtype=torch.int32, device=dev) for _ in range(P)]
+        gd, md = torch.from_numpy(g).to(dev), torch.from_numpy(m).to(dev)
+        # two destinations as tensors, one as a raw address, the way a peer's buffer arrives
+        B.signum_momentum_pack_scatter(gd, md if with_m else None, d, beta, [bufs[0], bufs[1].data_ptr(), bufs[2]],
+                                       row, ldw)
+        torch.cuda.synchronize()
+        m_ref = m[:d].copy()
+        if with_m:
+            words = oracle.signum_momentum_pack(np.ascontiguousarray(g[:d]), m_ref, 1, d, beta)
+            got_m = md.cpu().numpy()
+            assert np.array_equal(got_m[:d].view(np.uint32), m_ref.view(np.uint32))
+            assert np.array_equal(got_m[d:].view(np.uint32), m[d:].view(np.uint32))      # elements >= d untouched
+        else:
+            words = oracle.sign_pack(np.ascontiguousarray(g[:d]), 1, d)
+        for b in bufs:
+            got = b.cpu().numpy().view(np.uint32)
+            assert np.array_equal(got[row, :W], words[:W])
+            assert np.all(got[row, W:] == np.uint32(0xDEADBEEF))                         # row padding never written
+            assert np.all(np.delete(got, row, axis=0) == np.uint32(0xDEADBEEF))           # other workers' rows untouched
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("world,d,momentum", [(2, 100_003, True), (8, 1_000_003, True), (8, 70_001, False),
+                                             (3, 4_200_000, True)])
+def test_emulated_ranks_on_one_gpu_match_the_oracle(world, d, momentum):
+    """Every emulated rank owns its buffers on cuda:0; the rows travel by plain device copies (the
+    stand-in for the all-gather), so each rank's vote kernel reads only its own gathered copy."""
+    from paper_1802_04434_b200 import binding as B
+    B.lib()
+    run_emulated_ranks(world, d, momentum, "allgather", torch.device("cuda", 0))
+
+
+_SINGLE_RANK_P2P = r"""
+import os, sys
+sys.path.insert(0, {root!r}); sys.path.insert(0, {tests!r})
+import numpy as np, torch, torch.distributed as dist
+import oracle
+from paper_1802_04434_b200 import multi
+from test_worker_per_rank import worker_inputs, reference_run
+dev = torch.device("cuda", 0)
+torch.cuda.set_device(dev)
+multi.init(dev)
+try:
+    ws = multi.WorkerStep(70_001, dev, exchange="p2p")
+except Exception as e:                     # symmetric memory not available on this machine
+    print("NO-SYMMETRIC-MEMORY", repr(e)[:300]); multi.finish(); sys.exit(0)
+d, steps = 70_001, 3
+x0, g, m0 = worker_inputs(1, d, steps, seed=11)
+x, m = torch.from_numpy(x0.copy()).to(dev), torch.from_numpy(m0.copy()).to(dev)
+for k in range(steps):
+    ws.step(x, torch.from_numpy(g[k].copy()).to(dev), m, 0.9, 1e-3)
+torch.cuda.synchronize()
+ref, x_ref, m_ref = reference_run(x0, g, m0, d, 0.9, 1e-3)
+assert np.array_equal(x.cpu().numpy().view(np.uint32), x_ref.view(np.uint32))
+assert np.array_equal(m.cpu().numpy().reshape(-1).view(np.uint32), m_ref.view(np.uint32))
+assert np.array_equal(ws.vote.cpu().numpy().view(np.uint32), ref[-1][1])
+print("P2P-OK")
+multi.finish()
+"""
+
+
+@pytest.mark.gpu
+def test_p2p_transport_through_symmetric_memory_with_one_rank():
+    """The real plumbing of the p2p transport (NCCL group, symmetric-memory rendezvous, its barrier) with a world
+    of one rank, which is all one GPU allows: the peer table then holds only this GPU's own buffer."""
+    import subprocess
+    env = dict(os.environ, RANK="0", LOCAL_RANK="0", WORLD_SIZE="1", MASTER_ADDR="127.0.0.1",
+               MASTER_PORT=str(_free_port()))
+    code = _SINGLE_RANK_P2P.format(root=os.path.dirname(HERE), tests=HERE)
+    out = subprocess.run([sys.executable, "-c", code], capture_output=True, text=True, timeout=600, env=env)
+    assert out.returncode == 0, out.stdout[-2000:] + out.stderr[-3000:]
+    if "NO-SYMMETRIC-MEMORY" in out.stdout:
+        pytest.skip("torch symmetric memory is not available here: " + out.stdout.strip()[-300:])
+    assert "P2P-OK" in out.stdout
