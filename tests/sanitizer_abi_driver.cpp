@@ -72,6 +72,14 @@ int main() {
   EXPECT(ssgd_signsgd_step_noalloc(F, F, F, 1024, huge - 200, huge - 203, 0.9f, 0.1f, nullptr), SSGD_ERR_SCRATCH);
   EXPECT(ssgd_signsgd_step_noalloc(F, F, F, 1, huge - 100, huge - 103, 0.9f, 0.1f, nullptr), SSGD_ERR_SIZE);
 
+  uint32_t* rows[3] = {U, U + 1024, U + 2048};
+  uint32_t* rows_null[3] = {U, nullptr, U};
+  EXPECT(ssgd_signum_momentum_pack_scatter(F, F, 64, 0.9f, rows, 65, 0, 4, nullptr), SSGD_ERR_SIZE);
+  EXPECT(ssgd_signum_momentum_pack_scatter(F, F, 64, 0.9f, rows, 3, 1024, 4, nullptr), SSGD_ERR_SIZE);
+  EXPECT(ssgd_signum_momentum_pack_scatter(F, F, 64, 0.9f, rows, 3, 1023, huge / 4 * 4, nullptr), SSGD_ERR_SIZE);
+  EXPECT(ssgd_signum_momentum_pack_scatter(F, F, 64, 0.9f, rows_null, 3, 0, 4, nullptr), SSGD_ERR_NULL);
+  EXPECT(ssgd_signum_momentum_pack_scatter(F, nullptr, 0, 0.0f, rows, 3, 7, 0, nullptr), SSGD_OK);
+
   EXPECT(ssgd_warmup_steps(0.9f), 54);
   EXPECT(ssgd_warmup_steps(0.0f), 1);
   EXPECT(ssgd_warmup_steps(nan), 0);

@@ -118,6 +118,26 @@ def test_noalloc_step_rejects_before_touching_the_device(L):
     assert b"scratch" in L.ssgd_status_str(6)
 
 
+def test_pack_scatter_argument_checks(L):
+    f = L.ssgd_signum_momentum_pack_scatter
+    rows = (ctypes.c_void_p * 3)(A, A + 0x1000, A + 0x2000)
+    assert f(None, A, 64, 0.9, rows, 3, 0, 4, None) == NULL
+    assert f(A, A, 64, 0.9, None, 3, 0, 4, None) == NULL
+    assert f(A, None, 64, 0.9, rows, 3, 0, 4, None) == NULL            # m required when beta > 0
+    assert f(A, A + 4, 64, 0.9, rows, 3, 0, 4, None) == ALIGN
+    assert f(A, A, 64, 1.0, rows, 3, 0, 4, None) == ARG
+    assert f(A, A, 64, 0.9, rows, 0, 0, 4, None) == SIZE               # no destination
+    assert f(A, A, 64, 0.9, rows, 65, 0, 4, None) == SIZE              # more than SSGD_MAX_PEERS
+    assert f(A, A, 64, 0.9, rows, 3, 1024, 4, None) == SIZE            # row index out of range
+    assert f(A, A, 640, 0.9, rows, 3, 0, 16, None) == SIZE             # ldw < W
+    assert f(A, A, 64, 0.9, rows, 3, 0, 6, None) == ALIGN
+    bad = (ctypes.c_void_p * 3)(A, None, A)
+    assert f(A, A, 64, 0.9, bad, 3, 0, 4, None) == NULL
+    odd = (ctypes.c_void_p * 3)(A, A + 8, A)
+    assert f(A, A, 64, 0.9, odd, 3, 0, 4, None) == ALIGN
+    assert f(A, None, 0, 0.0, rows, 3, 5, 0, None) == OK               # d = 0; m optional when beta = 0
+
+
 def test_warmup_steps_is_host_arithmetic(L):
     assert L.ssgd_warmup_steps(0.9) == 54          # the value Theorem 3 prints for beta = 0.9
     assert L.ssgd_warmup_steps(0.0) == 1
