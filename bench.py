@@ -42,14 +42,14 @@ FALLBACK_HBM_GBS = 6650.0
 # captures summarised in profiles/ (taken at a reduced d with the same M and kernels; the path is
 # elementwise, so traffic grows in proportion to d).  Valid only while the kernel sources are unchanged.
 NCU_TRAFFIC = {
-    "source_sha256": "14fc0fb97f57511dbb3fe65a3c20fe277d739ec90ed0f5372787283f4173ece0",
+    "source_sha256": "af53dee7a9e6e3f6abcc1924996a3536224d2db4a641aadf25a3ce8723d581fc",
     "per_param": {
         # profiles/worker_vote_apply_kernels_d2p25_M16_ncu_full.md
-        "worker_pack_kernel:M16": {"bytes_per_param": (4.295064e9 + 2.164399e9) / 33554432, "d": 33554432},
-        "vote_kernel:M16": {"bytes_per_param": (67.118e6 + 0.771e6) / 33554432, "d": 33554432},
+        "worker_pack_kernel:M16": {"bytes_per_param": (4.294976e9 + 2.164599e9) / 33554432, "d": 33554432},
+        "vote_kernel:M16": {"bytes_per_param": (67.119e6 + 0.816e6) / 33554432, "d": 33554432},
         # (apply_kernel: in the reduced capture x is partly L2-resident, so its traffic does not scale with d)
         # profiles/fused_step_kernel_resnet50_M7_ncu_full.md (captured at full size)
-        "fused_step_kernel:M7": {"bytes_per_param": (1.533690e9 + 793.246464e6) / 25557056, "d": 25557056},
+        "fused_step_kernel:M7": {"bytes_per_param": (1.533629e9 + 793.557504e6) / 25557056, "d": 25557056},
     },
 }
 
@@ -81,7 +81,9 @@ def ncu_traffic(kernel: str, M: int, d: int):
     rec = NCU_TRAFFIC["per_param"].get("%s:M%d" % (kernel, M))
     if rec is None:
         return None, "no ncu capture of this kernel at this M"
-    return rec["bytes_per_param"] * d, "scaled by d from the capture at d = %d" % rec["d"]
+    if rec["d"] == d:
+        return rec["bytes_per_param"] * d, "ncu capture at this size"
+    return rec["bytes_per_param"] * d, "scaled by d from the ncu capture at d = %d" % rec["d"]
 
 
 def measured_peak():
