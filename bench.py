@@ -553,6 +553,8 @@ def run_ours(args):
         "gpu_launches": K * len(entries),
         "clocks": sampler.summary(clock_note),
     }
+    if not fused and d % 512 != 0:
+        line["gpu_launches_note"] = "plus one-warp tail launches per step (d is not a multiple of the 512-element span)"
     if world == 1 and not args.no_extra_kernels and not fused:
         # the fused kernel (the path for M <= 8) as one more entry, on the Resnet-50-sized workload
         del b, step
