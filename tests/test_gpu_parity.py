@@ -431,6 +431,33 @@ def test_resume_from_copied_state_is_bit_identical():
     assert torch.equal(xa, xb) and torch.equal(ma, mb)
 
 
+@pytest.mark.parametrize("M,d", [(5, 300_001), (12, 600_007)])
+def test_step_replayed_from_a_cuda_graph(M, d):
+    """The step entry point allocates nothing and never synchronises, so a caller can capture it into a CUDA
+    graph (one fused kernel for M = 5; worker + tail + vote + apply launches for M = 12) and replay it."""
+    cfg = wl.small_signum(d=d, M=M)
+    ld, ldw, W = cfg.ld, cfg.ldw, cfg.words
+    mu = cfg.shared(DEV)
+    xd, md = cfg.x0(DEV), cfg.m0(DEV)
+    gd = cfg.g(0, DEV, mu)
+    bits = torch.zeros(M, ldw, dtype=torch.int32, device=DEV)
+    vote = torch.zeros(W, dtype=torch.int32, device=DEV)
+    x_ref, m_ref = f32(xd).copy(), f32(md).reshape(-1).copy()
+    B.signsgd_step(xd.clone(), gd, md.clone(), M, d, ld, cfg.beta, cfg.delta, bits, ldw, vote)   # warm-up outside the capture
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        B.signsgd_step(xd, gd, md, M, d, ld, cfg.beta, cfg.delta, bits, ldw, vote)
+    for k in range(3):                                   # three replays = three steps on fresh gradients
+        gd.copy_(cfg.g(k, DEV, mu))
+        graph.replay()
+        torch.cuda.synchronize()
+        b_ref, v_ref = oracle.signsgd_step(x_ref, f32(gd).reshape(-1), m_ref, M, d, cfg.beta, cfg.delta, ld=ld, ldw=ldw)
+        assert np.array_equal(u32(bits).reshape(-1), b_ref) and np.array_equal(u32(vote), v_ref)
+        assert_same_f32(f32(xd), x_ref, "x, replay %d" % k)
+        assert_same_f32(f32(md).reshape(-1), m_ref, "m, replay %d" % k)
+
+
 # ------------------------------------------------------------------ Theorem 3 warm-up
 
 def test_warmup_length_matches_oracle():
