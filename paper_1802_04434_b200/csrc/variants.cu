@@ -16,34 +16,65 @@ namespace {
 // multiply-add per element, x <- fma(-delta, float(2P - M), x).  Lane layout as
 // in the apply kernel; each lane reads its word of every count plane.
 
+constexpr int kApplyUnroll = 2;   // 128-bit loads of x in flight per thread, as in the apply kernel of the 1-bit path
+
+// the sum of the M signs for the four elements of a lane, from its nibble of every count plane
+template <int NP>
+__device__ __forceinline__ void signed_sums(const unsigned (&nib)[NP], unsigned M, float (&s)[4]) {
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    int P = 0;
+#pragma unroll
+    for (int p = 0; p < NP; ++p) P |= (int)((nib[p] >> k) & 1u) << p;
+    s[k] = (float)(2 * P - (int)M);
+  }
+}
+
+// One tile of kThreads * 4 * kApplyUnroll elements per CTA; lane layout as in the apply kernel.
 template <int NP>
 __global__ void __launch_bounds__(kThreads)
 sum_apply_kernel(float* __restrict__ x, const uint32_t* __restrict__ counts, unsigned M,
                  unsigned long long d, unsigned long long ldc, float delta) {
+  constexpr int UNROLL = kApplyUnroll;
+  constexpr unsigned long long TILE = (unsigned long long)kThreads * 4 * UNROLL;
+  constexpr unsigned SPAN = 128 * UNROLL;
   const unsigned lane = threadIdx.x & 31u;
-  const unsigned long long stride = (unsigned long long)gridDim.x * kThreads * 4;
+  const unsigned warp = threadIdx.x >> 5;
+  const unsigned shift = 4u * (lane & 7u);
   const float neg = -delta;
-  for (unsigned long long e = ((unsigned long long)blockIdx.x * kThreads + threadIdx.x) * 4; e < d; e += stride) {
-    const unsigned shift = 4u * (lane & 7u);        // e is a multiple of 4: (e % 32) = 4 (lane % 8)
-    unsigned nib[NP];
+  const unsigned long long e0 = (unsigned long long)blockIdx.x * TILE + (unsigned long long)warp * SPAN;
+  if (e0 >= d) return;
+  if (e0 + SPAN <= d) {
+    float4 xv[UNROLL];
+    unsigned nib[UNROLL][NP];
 #pragma unroll
-    for (int p = 0; p < NP; ++p) nib[p] = __ldg(counts + (unsigned long long)p * ldc + (e >> 5)) >> shift;
-    float s[4];
+    for (int u = 0; u < UNROLL; ++u) {
+      xv[u] = ld128(x + e0 + u * 128 + lane * 4);
 #pragma unroll
-    for (int k = 0; k < 4; ++k) {
-      int P = 0;
-#pragma unroll
-      for (int p = 0; p < NP; ++p) P |= (int)((nib[p] >> k) & 1u) << p;
-      s[k] = (float)(2 * P - (int)M);
+      for (int p = 0; p < NP; ++p)
+        nib[u][p] = __ldg(counts + (unsigned long long)p * ldc + (e0 >> 5) + u * 4 + (lane >> 3)) >> shift;
     }
-    if (e + 4 <= d) {
-      float4 v = ld128(x + e);
+#pragma unroll
+    for (int u = 0; u < UNROLL; ++u) {
+      float s[4];
+      signed_sums<NP>(nib[u], M, s);
+      float4 v = xv[u];
       v.x = __fmaf_rn(neg, s[0], v.x);
       v.y = __fmaf_rn(neg, s[1], v.y);
       v.z = __fmaf_rn(neg, s[2], v.z);
       v.w = __fmaf_rn(neg, s[3], v.w);
-      st128(x + e, v);
-    } else {
+      st128(x + e0 + u * 128 + lane * 4, v);
+    }
+  } else {
+#pragma unroll 1
+    for (int u = 0; u < UNROLL; ++u) {
+      const unsigned long long e = e0 + u * 128 + lane * 4;
+      if (e >= d) break;
+      unsigned nib[NP];
+#pragma unroll
+      for (int p = 0; p < NP; ++p) nib[p] = __ldg(counts + (unsigned long long)p * ldc + (e >> 5)) >> shift;
+      float s[4];
+      signed_sums<NP>(nib, M, s);
 #pragma unroll
       for (int k = 0; k < 4; ++k)
         if (e + k < d) x[e + k] = __fmaf_rn(neg, s[k], x[e + k]);
@@ -54,8 +85,8 @@ sum_apply_kernel(float* __restrict__ x, const uint32_t* __restrict__ counts, uns
 template <int NP>
 void launch_sum_apply_np(float* x, const uint32_t* counts, size_t M, size_t d, size_t ldc, float delta,
                          cudaStream_t s) {
-  const unsigned long long ctas = ((d + 3) / 4 + kThreads - 1) / kThreads;
-  sum_apply_kernel<NP><<<grid_for(ctas), kThreads, 0, s>>>(x, counts, (unsigned)M, d, ldc, delta);
+  constexpr unsigned long long TILE = (unsigned long long)kThreads * 4 * kApplyUnroll;
+  sum_apply_kernel<NP><<<grid_for((d + TILE - 1) / TILE), kThreads, 0, s>>>(x, counts, (unsigned)M, d, ldc, delta);
 }
 
 ssgd_status launch_sum_apply(float* x, const uint32_t* counts, size_t M, size_t d, size_t ldc,
@@ -95,85 +126,131 @@ __device__ __forceinline__ unsigned active_nibble(const float4& v, float tau) {
          ((fabsf(v.w) < tau) ? 0u : 8u);
 }
 
-// Same tiling as the worker kernel (one tile of kThreads * 16 elements of one row
-// per CTA, all loads of a thread issued before their first use), with a second
-// output plane.
+// One span that crosses the end of its row: element-wise guards; bits at
+// positions >= d stay 0, nothing at or beyond d is written.
 template <bool MOMENTUM>
-__global__ void __launch_bounds__(kThreads)
+__device__ __forceinline__ void ternary_ragged_span(const float* __restrict__ gr, float* __restrict__ mr,
+                                                    uint32_t* __restrict__ sr, uint32_t* __restrict__ ar,
+                                                    unsigned long long d, unsigned long long e0, float beta,
+                                                    float omb, float tau) {
+  const unsigned lane = threadIdx.x & 31u;
+#pragma unroll 1
+  for (int u = 0; u < kTernaryUnroll; ++u) {
+    const unsigned long long e = e0 + u * 128 + lane * 4;
+    unsigned snib = 0, anib = 0;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      if (e + k < d) {
+        float v = gr[e + k];
+        if (MOMENTUM) {
+          v = momentum_update(beta, omb, mr[e + k], v);
+          mr[e + k] = v;
+        }
+        snib |= sign_bit(v) << k;
+        anib |= ((fabsf(v) < tau) ? 0u : 1u) << k;
+      }
+    }
+    const unsigned sword = assemble_word(snib, lane);
+    const unsigned aword = assemble_word(anib, lane);
+    const unsigned long long first = e0 + u * 128 + (lane >> 3) * 32;  // first element of the word
+    if ((lane & 7u) == 0 && first < d) {
+      sr[u * 4 + (lane >> 3)] = sword;
+      ar[u * 4 + (lane >> 3)] = aword;
+    }
+  }
+}
+
+// Same tiling and structure as the worker kernel of the 1-bit path (grid x = tile
+// of kThreads * 16 elements within the row, y = row; all loads of a thread issued
+// before their first use; RAGGED = false leaves the last partial span of a row to
+// the tail kernel), with a second output plane.
+template <bool MOMENTUM, bool RAGGED>
+__global__ void __launch_bounds__(kThreads, 1)
 ternary_pack_kernel(const float* __restrict__ g, float* __restrict__ m,
                     uint32_t* __restrict__ sign_bits, uint32_t* __restrict__ active_bits,
                     unsigned long long d, unsigned long long ld, unsigned long long ldw,
-                    unsigned long long tiles_per_row, unsigned long long total_tiles,
                     float beta, float omb, float tau) {
   constexpr int UNROLL = kTernaryUnroll;
   constexpr unsigned long long TILE = (unsigned long long)kThreads * 4 * UNROLL;
   constexpr unsigned SPAN = 128 * UNROLL;
   const unsigned lane = threadIdx.x & 31u;
   const unsigned warp = threadIdx.x >> 5;
-  for (unsigned long long t = blockIdx.x; t < total_tiles; t += gridDim.x) {
-    const unsigned long long row = t / tiles_per_row;
-    const unsigned long long tile = t - row * tiles_per_row;
-    const unsigned long long e0 = tile * TILE + (unsigned long long)warp * SPAN;
-    if (e0 >= d) continue;
-    const float* gr = g + row * ld;
-    float* mr = MOMENTUM ? m + row * ld : nullptr;
-    uint32_t* sr = sign_bits + row * ldw + (e0 >> 5);
-    uint32_t* ar = active_bits + row * ldw + (e0 >> 5);
-    if (e0 + SPAN <= d) {
-      float4 gv[UNROLL], mv[UNROLL];
+  const unsigned long long row = blockIdx.y;
+  const unsigned long long e0 = (unsigned long long)blockIdx.x * TILE + (unsigned long long)warp * SPAN;
+  if (e0 + SPAN > d) {
+    if (RAGGED && e0 < d)
+      ternary_ragged_span<MOMENTUM>(g + row * ld, MOMENTUM ? m + row * ld : nullptr,
+                                    sign_bits + row * ldw + (e0 >> 5), active_bits + row * ldw + (e0 >> 5), d, e0,
+                                    beta, omb, tau);
+    return;
+  }
+  const float* gr = g + row * ld + e0 + lane * 4;
+  float* mr = MOMENTUM ? m + row * ld + e0 + lane * 4 : nullptr;
+  float4 gv[UNROLL], mv[UNROLL];
 #pragma unroll
-      for (int u = 0; u < UNROLL; ++u) gv[u] = ld128(gr + e0 + u * 128 + lane * 4);
-      if (MOMENTUM) {
+  for (int u = 0; u < UNROLL; ++u) gv[u] = ld128(gr + u * 128);
+  if (MOMENTUM) {
 #pragma unroll
-        for (int u = 0; u < UNROLL; ++u) mv[u] = ld128(mr + e0 + u * 128 + lane * 4);
-      }
-      unsigned smine = 0, amine = 0;
+    for (int u = 0; u < UNROLL; ++u) mv[u] = ld128(mr + u * 128);
+  }
+  unsigned smine = 0, amine = 0;
 #pragma unroll
-      for (int u = 0; u < UNROLL; ++u) {
-        float4 v = gv[u];
-        if (MOMENTUM) {
-          v = momentum_update4(beta, omb, mv[u], v);
-          st128(mr + e0 + u * 128 + lane * 4, v);
-        }
-        const unsigned sword = assemble_word(sign_nibble(v), lane);
-        const unsigned aword = assemble_word(active_nibble(v, tau), lane);
-        if ((lane & 7u) == (unsigned)u) {
-          smine = sword;
-          amine = aword;
-        }
-      }
-      if ((lane & 7u) < (unsigned)UNROLL) {
-        sr[own_word_index<UNROLL>(lane)] = smine;
-        ar[own_word_index<UNROLL>(lane)] = amine;
-      }
-    } else {
-      // ragged end of the row: element-wise guards; bits at positions >= d stay 0
-#pragma unroll 1
-      for (int u = 0; u < UNROLL; ++u) {
-        const unsigned long long e = e0 + u * 128 + lane * 4;
-        unsigned snib = 0, anib = 0;
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-          if (e + k < d) {
-            float v = gr[e + k];
-            if (MOMENTUM) {
-              v = momentum_update(beta, omb, mr[e + k], v);
-              mr[e + k] = v;
-            }
-            snib |= sign_bit(v) << k;
-            anib |= ((fabsf(v) < tau) ? 0u : 1u) << k;
-          }
-        }
-        const unsigned sword = assemble_word(snib, lane);
-        const unsigned aword = assemble_word(anib, lane);
-        const unsigned long long first = e0 + u * 128 + (lane >> 3) * 32;  // first element of the word
-        if ((lane & 7u) == 0 && first < d) {
-          sr[u * 4 + (lane >> 3)] = sword;
-          ar[u * 4 + (lane >> 3)] = aword;
-        }
-      }
+  for (int u = 0; u < UNROLL; ++u) {
+    float4 v = gv[u];
+    if (MOMENTUM) {
+      v = momentum_update4(beta, omb, mv[u], v);
+      st128(mr + u * 128, v);
+    }
+    const unsigned sword = assemble_word(sign_nibble(v), lane);
+    const unsigned aword = assemble_word(active_nibble(v, tau), lane);
+    if ((lane & 7u) == (unsigned)u) {
+      smine = sword;
+      amine = aword;
     }
   }
+  if ((lane & 7u) < (unsigned)UNROLL) {
+    const unsigned long long w = row * ldw + (e0 >> 5) + own_word_index<UNROLL>(lane);
+    sign_bits[w] = smine;
+    active_bits[w] = amine;
+  }
+}
+
+template <bool MOMENTUM>
+__global__ void __launch_bounds__(32)
+ternary_tail_kernel(const float* __restrict__ g, float* __restrict__ m, uint32_t* __restrict__ sign_bits,
+                    uint32_t* __restrict__ active_bits, unsigned long long d, unsigned long long ld,
+                    unsigned long long ldw, float beta, float omb, float tau) {
+  constexpr unsigned SPAN = 128 * kTernaryUnroll;
+  const unsigned long long row = blockIdx.x;
+  const unsigned long long e0 = d / SPAN * SPAN;
+  if (e0 < d)
+    ternary_ragged_span<MOMENTUM>(g + row * ld, MOMENTUM ? m + row * ld : nullptr, sign_bits + row * ldw + (e0 >> 5),
+                                  active_bits + row * ldw + (e0 >> 5), d, e0, beta, omb, tau);
+}
+
+// Large inputs (at least 8 CTAs per SM): interior-only main kernel, with the unused shared-memory request
+// that the worker kernel of the 1-bit path uses as a carve-out hint, plus a one-warp-per-row tail launch
+// when d is not a multiple of the span; smaller inputs: one launch with the guarded path inline.
+template <bool MOMENTUM>
+ssgd_status launch_ternary_pack(const float* g, float* m, size_t M, size_t d, size_t ld, float beta, float tau,
+                                uint32_t* sign_bits, uint32_t* active_bits, size_t ldw, cudaStream_t s) {
+  constexpr unsigned long long TILE = (unsigned long long)kThreads * 4 * kTernaryUnroll;
+  DeviceInfo di;
+  if (!device_info(&di)) return SSGD_ERR_CUDA;
+  const unsigned long long tiles_per_row = (d + TILE - 1) / TILE;
+  if (tiles_per_row > kMaxGrid) return SSGD_ERR_SIZE;
+  const dim3 grid((unsigned)tiles_per_row, (unsigned)M);
+  const float omb = 1.0f - beta;
+  if (tiles_per_row * M >= 8ull * di.sms) {
+    ternary_pack_kernel<MOMENTUM, false><<<grid, kThreads, 36 * 1024, s>>>(g, m, sign_bits, active_bits, d, ld, ldw,
+                                                                             beta, omb, tau);
+    if (d % (128 * kTernaryUnroll) != 0)
+      ternary_tail_kernel<MOMENTUM><<<(unsigned)M, 32, 0, s>>>(g, m, sign_bits, active_bits, d, ld, ldw, beta, omb, tau);
+  } else {
+    ternary_pack_kernel<MOMENTUM, true><<<grid, kThreads, 0, s>>>(g, m, sign_bits, active_bits, d, ld, ldw, beta, omb,
+                                                                  tau);
+  }
+  return launch_status();
 }
 
 // [D >= T] per bit position for a bit-sliced D held in NP planes (D < 2^NP):
@@ -222,24 +299,46 @@ quorum_vote_kernel(const uint32_t* __restrict__ sign_bits, const uint32_t* __res
   }
 }
 
+__device__ __forceinline__ float4 ternary_apply4(float4 v, unsigned snib, unsigned anib, float delta, float minus) {
+  if (anib & 1u) v.x = __fadd_rn(v.x, (snib & 1u) ? minus : delta);
+  if (anib & 2u) v.y = __fadd_rn(v.y, (snib & 2u) ? minus : delta);
+  if (anib & 4u) v.z = __fadd_rn(v.z, (snib & 4u) ? minus : delta);
+  if (anib & 8u) v.w = __fadd_rn(v.w, (snib & 8u) ? minus : delta);
+  return v;
+}
+
+// One tile of kThreads * 4 * kApplyUnroll elements per CTA; lane layout as in the apply kernel.
 __global__ void __launch_bounds__(kThreads)
 ternary_apply_kernel(float* __restrict__ x, const uint32_t* __restrict__ vote_sign,
                      const uint32_t* __restrict__ vote_active, unsigned long long d, float delta) {
+  constexpr int UNROLL = kApplyUnroll;
+  constexpr unsigned long long TILE = (unsigned long long)kThreads * 4 * UNROLL;
+  constexpr unsigned SPAN = 128 * UNROLL;
   const unsigned lane = threadIdx.x & 31u;
-  const unsigned long long stride = (unsigned long long)gridDim.x * kThreads * 4;
+  const unsigned warp = threadIdx.x >> 5;
+  const unsigned shift = 4u * (lane & 7u);
   const float minus = -delta;
-  for (unsigned long long e = ((unsigned long long)blockIdx.x * kThreads + threadIdx.x) * 4; e < d; e += stride) {
-    const unsigned shift = 4u * (lane & 7u);
-    const unsigned snib = __ldg(vote_sign + (e >> 5)) >> shift;
-    const unsigned anib = __ldg(vote_active + (e >> 5)) >> shift;
-    if (e + 4 <= d) {
-      float4 v = ld128(x + e);
-      if (anib & 1u) v.x = __fadd_rn(v.x, (snib & 1u) ? minus : delta);
-      if (anib & 2u) v.y = __fadd_rn(v.y, (snib & 2u) ? minus : delta);
-      if (anib & 4u) v.z = __fadd_rn(v.z, (snib & 4u) ? minus : delta);
-      if (anib & 8u) v.w = __fadd_rn(v.w, (snib & 8u) ? minus : delta);
-      st128(x + e, v);
-    } else {
+  const unsigned long long e0 = (unsigned long long)blockIdx.x * TILE + (unsigned long long)warp * SPAN;
+  if (e0 >= d) return;
+  if (e0 + SPAN <= d) {
+    float4 xv[UNROLL];
+    unsigned sn[UNROLL], an[UNROLL];
+#pragma unroll
+    for (int u = 0; u < UNROLL; ++u) {
+      xv[u] = ld128(x + e0 + u * 128 + lane * 4);
+      sn[u] = __ldg(vote_sign + (e0 >> 5) + u * 4 + (lane >> 3)) >> shift;
+      an[u] = __ldg(vote_active + (e0 >> 5) + u * 4 + (lane >> 3)) >> shift;
+    }
+#pragma unroll
+    for (int u = 0; u < UNROLL; ++u)
+      st128(x + e0 + u * 128 + lane * 4, ternary_apply4(xv[u], sn[u], an[u], delta, minus));
+  } else {
+#pragma unroll 1
+    for (int u = 0; u < UNROLL; ++u) {
+      const unsigned long long e = e0 + u * 128 + lane * 4;
+      if (e >= d) break;
+      const unsigned snib = __ldg(vote_sign + (e >> 5)) >> shift;
+      const unsigned anib = __ldg(vote_active + (e >> 5)) >> shift;
 #pragma unroll
       for (int k = 0; k < 4; ++k)
         if (e + k < d && ((anib >> k) & 1u)) x[e + k] = __fadd_rn(x[e + k], ((snib >> k) & 1u) ? minus : delta);
@@ -281,6 +380,7 @@ ssgd_status ssgd_sum_apply(float* x, const uint32_t* counts, size_t M, size_t d,
   if (st != SSGD_OK) return st;
   if (!isfinite(delta)) return SSGD_ERR_ARG;
   if (d == 0) return SSGD_OK;
+  if (d / ((size_t)kThreads * 4 * kApplyUnroll) >= kMaxGrid) return SSGD_ERR_SIZE;   // beyond any device's memory
   return launch_sum_apply(x, counts, M, d, ldc, delta, static_cast<cudaStream_t>(stream));
 }
 
@@ -295,17 +395,9 @@ ssgd_status ssgd_ternary_pack(const float* g, float* m, size_t M, size_t d, size
   if (!beta_ok(beta) || !(tau >= 0.0f) || !isfinite(tau)) return SSGD_ERR_ARG;
   if (!m && beta != 0.0f) return SSGD_ERR_NULL;
   if (d == 0) return SSGD_OK;
-  constexpr unsigned long long TILE = (unsigned long long)kThreads * 4 * kTernaryUnroll;
-  const unsigned long long tiles_per_row = (d + TILE - 1) / TILE;
-  const unsigned long long total = tiles_per_row * M;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  if (m)
-    ternary_pack_kernel<true><<<grid_for(total), kThreads, 0, s>>>(g, m, sign_bits, active_bits, d, ld, ldw,
-                                                                   tiles_per_row, total, beta, 1.0f - beta, tau);
-  else
-    ternary_pack_kernel<false><<<grid_for(total), kThreads, 0, s>>>(g, nullptr, sign_bits, active_bits, d, ld,
-                                                                    ldw, tiles_per_row, total, 0.0f, 1.0f, tau);
-  return launch_status();
+  return m ? launch_ternary_pack<true>(g, m, M, d, ld, beta, tau, sign_bits, active_bits, ldw, s)
+           : launch_ternary_pack<false>(g, nullptr, M, d, ld, 0.0f, tau, sign_bits, active_bits, ldw, s);
 }
 
 ssgd_status ssgd_quorum_vote(const uint32_t* sign_bits, const uint32_t* active_bits, size_t M, size_t d,
@@ -346,9 +438,10 @@ ssgd_status ssgd_ternary_apply(float* x, const uint32_t* vote_sign, const uint32
   if (d > SIZE_MAX - 31) return SSGD_ERR_SIZE;
   if (!isfinite(delta)) return SSGD_ERR_ARG;
   if (d == 0) return SSGD_OK;
-  const unsigned long long ctas = ((d + 3) / 4 + kThreads - 1) / kThreads;
-  ternary_apply_kernel<<<grid_for(ctas), kThreads, 0, static_cast<cudaStream_t>(stream)>>>(x, vote_sign, vote_active,
-                                                                                          d, delta);
+  constexpr unsigned long long TILE = (unsigned long long)kThreads * 4 * kApplyUnroll;
+  if (d / TILE >= kMaxGrid) return SSGD_ERR_SIZE;   // beyond any device's memory
+  ternary_apply_kernel<<<grid_for((d + TILE - 1) / TILE), kThreads, 0, static_cast<cudaStream_t>(stream)>>>(
+      x, vote_sign, vote_active, d, delta);
   return launch_status();
 }
 

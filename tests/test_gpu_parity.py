@@ -585,6 +585,41 @@ def test_abstention_path(M):
             assert_same_f32(f32(xd), x_ref, "x")
 
 
+@pytest.mark.parametrize("M,d,with_m", [(8, 1_000_003, True), (3, 2_500_003, False)])
+def test_abstention_path_large_odd_d(M, d, with_m):
+    # large enough for the interior-only ternary pack kernel and its tail launch; rows longer than d
+    ld, W = wl.round_up(d, 4) + 8, oracle.words(d)
+    ldw = wl.round_up(W, 4) + 4
+    g, m, x = big_inputs(M, d, ld, seed=M * 17 + d % 1000, with_m=with_m)
+    beta, tau, Q = (0.9, 0.2, 2) if with_m else (0.0, 0.5, 1)
+    gd, xd = torch.from_numpy(g).to(DEV), torch.from_numpy(x).to(DEV)
+    md = torch.from_numpy(m).to(DEV) if with_m else None
+    sb = torch.full((M, ldw), CANARY_WORD, dtype=torch.int32, device=DEV)
+    ab = torch.full((M, ldw), CANARY_WORD, dtype=torch.int32, device=DEV)
+    B.ternary_pack(gd, md, M, d, ld, beta, tau, sb, ab, ldw)
+    m_ref = m.copy().reshape(-1) if with_m else None
+    sb_ref, ab_ref = oracle.ternary_pack(g.reshape(-1), m_ref, M, d, beta, tau, ld=ld, ldw=ldw)
+    check_rows(sb, sb_ref, M, ldw, W, "sign plane")
+    check_rows(ab, ab_ref, M, ldw, W, "active plane")
+    if with_m:
+        gm = f32(md)
+        assert_same_f32(gm.reshape(-1), m_ref, "m")
+        assert np.array_equal(gm[:, d:].view(np.uint32), m[:, d:].view(np.uint32))
+    sb[:, W:] = 0
+    ab[:, W:] = 0
+    vs = torch.full((W + 4,), CANARY_WORD, dtype=torch.int32, device=DEV)
+    va = torch.full((W + 4,), CANARY_WORD, dtype=torch.int32, device=DEV)
+    B.quorum_vote(sb, ab, M, d, ldw, Q, vs, va)
+    vs_ref, va_ref = oracle.quorum_vote(u32(sb).reshape(-1).copy(), u32(ab).reshape(-1).copy(), M, d, Q, ldw=ldw)
+    assert np.array_equal(u32(vs)[:W], vs_ref) and np.array_equal(u32(va)[:W], va_ref)
+    B.ternary_apply(xd, vs, va, d, 1e-3)
+    x_ref = x[:d].copy()
+    oracle.ternary_apply(x_ref, vs_ref, va_ref, d, 1e-3)
+    gx = f32(xd)
+    assert_same_f32(gx[:d], x_ref, "x")
+    assert np.all(gx[d:] == np.float32(CANARY_F))
+
+
 # ------------------------------------------------------------------ Section 3: density and Welford
 
 @pytest.mark.parametrize("d", [1, 3, 1000, 4099, 1 << 20, (1 << 22) + 5])
