@@ -227,6 +227,27 @@ ssgd_status ssgd_signsgd_step_host(float* x, const float* g_host, float* m,
                                    uint32_t* vote_ws, uint32_t* vote_host,
                                    void* stream);
 
+/* ssgd_majority_vote (Algorithm 3, server block) computed by a second kernel design: the M rows of a
+ * 1024-word tile are staged through shared memory by bulk asynchronous copies (8 rows per mbarrier
+ * phase, double-buffered) instead of being loaded into registers directly.  Same arguments, same
+ * output words.  It is kept so that the two designs can be measured side by side (on B200 the direct
+ * kernel is at least as fast; the step entry points use that one).
+ *   status  in/out DEVICE unsigned (4-byte aligned), set it to 0 before the call: every wait in the
+ *                  kernel has an iteration limit, and a CTA whose copies do not arrive within it
+ *                  sets bit 0 here and writes no output instead of waiting forever.  Read it after
+ *                  synchronising the stream; it stays 0 in normal operation. */
+ssgd_status ssgd_majority_vote_staged(const uint32_t* bits, size_t M, size_t d,
+                                      size_t ldw, uint32_t* vote, unsigned* status,
+                                      void* stream);
+
+/* Self-test of the bounded waits of ssgd_majority_vote_staged (no counterpart in the paper): the same
+ * launch with every wait made to run out (each phase is armed for more bytes than its copies deliver;
+ * all copies still complete).  The kernel must return within its iteration limits (about 0.2 s) with
+ * bit 0 of *status set and `vote` untouched; the context stays usable.  d <= 32768 (one tile). */
+ssgd_status ssgd_majority_vote_staged_wait_selftest(const uint32_t* bits, size_t M, size_t d,
+                                                    size_t ldw, uint32_t* vote,
+                                                    unsigned* status, void* stream);
+
 /* Most ranks one ssgd_signum_momentum_pack_scatter call can send to. */
 #define SSGD_MAX_PEERS 64
 

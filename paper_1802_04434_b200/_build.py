@@ -7,7 +7,7 @@ import subprocess
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(_HERE)
-SOURCES = [os.path.join(_HERE, "csrc", n) for n in ("signsgd.cu", "variants.cu", "stats.cu", "exchange.cu")]
+SOURCES = [os.path.join(_HERE, "csrc", n) for n in ("signsgd.cu", "variants.cu", "stats.cu", "exchange.cu", "vote_staged.cu")]
 HEADERS = [os.path.join(ROOT, "include", "signsgd.h")] + [
     os.path.join(_HERE, "csrc", n) for n in ("device_common.cuh", "host_common.h")]
 LIB = os.path.join(_HERE, "libsignsgd_b200.so")

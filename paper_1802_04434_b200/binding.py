@@ -68,6 +68,8 @@ def lib() -> ctypes.CDLL:
         "ssgd_signsgd_step_host": [vp, vp, vp, sz, sz, sz, f32, f32, vp, vp, sz, vp, vp, vp],
         "ssgd_signsgd_step_noalloc": [vp, vp, vp, sz, sz, sz, f32, f32, vp],
         "ssgd_signum_momentum_pack_scatter": [vp, vp, sz, f32, vp, sz, sz, sz, vp],
+        "ssgd_majority_vote_staged": [vp, sz, sz, sz, vp, vp, vp],
+        "ssgd_majority_vote_staged_wait_selftest": [vp, sz, sz, sz, vp, vp, vp],
     }
     for name, args in sigs.items():
         fn = getattr(L, name)
@@ -144,6 +146,17 @@ def majority_vote(bits: torch.Tensor, M: int, d: int, ldw: int, vote: torch.Tens
     _check(lib().ssgd_majority_vote(_ptr(bits, WORD_DTYPE, "bits"), M, d, ldw,
                                     _ptr(vote, WORD_DTYPE, "vote"), _stream(stream)),
            "ssgd_majority_vote")
+
+
+def majority_vote_staged(bits: torch.Tensor, M: int, d: int, ldw: int, vote: torch.Tensor, status: torch.Tensor,
+                         stream=None) -> None:
+    """The majority vote by the kernel that stages the rows through shared memory with bulk copies; same
+    output as `majority_vote`.  `status` is a one-element int32 device tensor, zero before the call; it is
+    non-zero afterwards only if a bounded wait in the kernel ran out."""
+    _need(bits, M * ldw, "bits"); _need(vote, -(-d // 32), "vote"); _need(status, 1, "status")
+    _check(lib().ssgd_majority_vote_staged(_ptr(bits, WORD_DTYPE, "bits"), M, d, ldw, _ptr(vote, WORD_DTYPE, "vote"),
+                                           _ptr(status, torch.int32, "status"), _stream(stream)),
+           "ssgd_majority_vote_staged")
 
 
 def sign_apply(x: torch.Tensor, vote: torch.Tensor, d: int, delta: float, stream=None) -> None:

@@ -4,8 +4,8 @@
                     [--reps 20] [--out sweep.tsv]
 
 For every point and every kernel of the step (worker momentum + pack, majority vote, apply) and for
-the whole step (and, as a yardstick for the short vote kernel, for a plain device copy of the vote's
-byte volume), prints the time per launch, the algorithmic GB/s and its fraction of the measured
+the whole step (and, beside the vote kernel, for its shared-memory-staged alternative and for a plain
+device copy of the vote's byte volume as a yardstick), prints the time per launch, the algorithmic GB/s and its fraction of the measured
 copy peak.  Launches are replayed from a CUDA graph between two CUDA events.  When
 one launch touches less than twice the L2 size, the launches rotate over several buffer sets so that
 the combined footprint exceeds it (column `cold` = 1); for the smallest sizes that would need more
@@ -106,6 +106,12 @@ def run_point(d: int, M: int, reps: int, dev) -> list:
     rec("momentum_pack", ms, bytes_worker, n_sets_big * bytes_worker >= 2 * L2_BYTES)
     ms = time_launches(lambda s: B.majority_vote(bits[s], M, d, ldw, vote[s]), n_sets, reps)
     rec("majority_vote", ms, bytes_vote, n_sets * bytes_vote >= 2 * L2_BYTES)
+    # the other vote kernel design: rows staged through shared memory by bulk copies
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    ms = time_launches(lambda s: B.majority_vote_staged(bits[s], M, d, ldw, vote[s], status), n_sets, reps)
+    rec("majority_vote_staged", ms, bytes_vote, n_sets * bytes_vote >= 2 * L2_BYTES)
+    if int(status.item()) != 0:
+        raise SystemExit("a bounded wait of the staged vote kernel ran out")
     # yardstick for the short vote kernel: a plain device copy that moves the same number of bytes.
     # Sources and destinations are separate buffers and both rotate, so no launch reads what an
     # earlier one left in L2.

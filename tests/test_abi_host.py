@@ -85,6 +85,17 @@ def test_vote_argument_checks(L):
     assert f(A, 3, 0, 0, A, None) == OK
 
 
+def test_staged_vote_argument_checks(L):
+    for f in (L.ssgd_majority_vote_staged, L.ssgd_majority_vote_staged_wait_selftest):
+        assert f(None, 3, 64, 4, A, A, None) == NULL
+        assert f(A, 3, 64, 4, A, None, None) == NULL           # the status word is required
+        assert f(A, 3, 64, 4, A, A + 2, None) == ALIGN
+        assert f(A, 3, 64, 6, A, A, None) == ALIGN
+        assert f(A, 0, 64, 4, A, A, None) == SIZE
+        assert f(A, 3, 0, 0, A, A, None) == OK
+    assert L.ssgd_majority_vote_staged_wait_selftest(A, 3, 1 << 20, 1 << 15, A, A, None) == SIZE
+
+
 def test_apply_argument_checks(L):
     f = L.ssgd_sign_apply
     assert f(None, A, 64, 0.1, None) == NULL

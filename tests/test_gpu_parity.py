@@ -113,6 +113,56 @@ def test_majority_vote_small(M):
         assert np.all(got[W:] == np.uint32(0xDEADBEEF))
 
 
+@pytest.mark.parametrize("M", [1, 2, 3, 7, 8, 9, 16, 17, 31, 33, 100, 1024])
+def test_majority_vote_staged_through_shared_memory(M):
+    # the second kernel design (rows staged by bulk copies, 8 rows per mbarrier phase): same words
+    for d in (1, 33, 4097, 32768, 32768 + 5, 100_003 if M <= 100 else 40_000, 1_000_003 if M <= 17 else 70_001):
+        r = np.random.default_rng(M * 1000 + d)
+        W = oracle.words(d)
+        ldw = wl.round_up(W, 4) + (4 if M % 2 else 0)
+        s = (r.random((M, d)) < r.random(d)).astype(np.uint8) if M * d <= 20_000_000 else \
+            (r.random((M, d), dtype=np.float32) < 0.5).astype(np.uint8)
+        rows = np.zeros((M, ldw), dtype=np.uint32)
+        for w in range(M):
+            rows[w, :W] = oracle.pack_bits(s[w])
+        rows[:, W:] = r.integers(0, 2**32, size=(M, ldw - W), dtype=np.uint32)   # garbage in row padding
+        vote = torch.full((W + 4,), CANARY_WORD, dtype=torch.int32, device=DEV)
+        status = torch.zeros(1, dtype=torch.int32, device=DEV)
+        B.majority_vote_staged(torch.from_numpy(rows.view(np.int32)).to(DEV), M, d, ldw, vote, status)
+        ref = oracle.majority_vote(rows.reshape(-1), M, d, ldw=ldw)
+        got = u32(vote)
+        assert int(status.item()) == 0
+        assert np.array_equal(got[:W], ref), "M=%d d=%d" % (M, d)
+        assert np.all(got[W:] == np.uint32(0xDEADBEEF))
+
+
+def test_staged_vote_bounded_waits_run_out_and_report():
+    """Every wait in the staged kernel has an iteration limit.  The self-test entry arms each phase for more
+    bytes than its copies deliver, so the waits must run out: the call returns, the status word says so, the
+    output is untouched, and the device is fine afterwards."""
+    M, d = 19, 20_000
+    W = oracle.words(d)
+    ldw = wl.round_up(W, 4)
+    bits = torch.randint(-2**31, 2**31 - 1, (M, ldw), dtype=torch.int32, device=DEV)
+    vote = torch.full((W,), CANARY_WORD, dtype=torch.int32, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    L = B.lib()
+    rc = L.ssgd_majority_vote_staged_wait_selftest(bits.data_ptr(), M, d, ldw, vote.data_ptr(), status.data_ptr(),
+                                                   torch.cuda.current_stream().cuda_stream)
+    assert rc == 0
+    torch.cuda.synchronize()
+    assert int(status.item()) == 1
+    assert np.all(u32(vote) == np.uint32(0xDEADBEEF))
+    assert L.ssgd_majority_vote_staged_wait_selftest(bits.data_ptr(), M, 1 << 20, 1 << 15, vote.data_ptr(),
+                                                     status.data_ptr(), None) == 3          # larger sizes refused
+    status.zero_()
+    B.majority_vote_staged(bits, M, d, ldw, vote, status)                                    # and it still works
+    ref = torch.zeros(W, dtype=torch.int32, device=DEV)
+    B.majority_vote(bits, M, d, ldw, ref)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0 and torch.equal(vote, ref)
+
+
 def test_majority_vote_ignores_garbage_padding_bits():
     # padding bits of the last word are the caller's to keep 0; the vote masks them anyway
     M, d = 3, 40

@@ -65,7 +65,7 @@ def test_host_argument_checks_are_clean_under_asan_and_ubsan(tmp_path):
            "-I", os.path.join(ROOT, "include"),
            "-Xcompiler", "-fsanitize=address", "-Xcompiler", "-fsanitize=undefined",
            "-Xcompiler", "-fno-sanitize-recover=all",
-           *[os.path.join(csrc, n) for n in ("signsgd.cu", "variants.cu", "stats.cu", "exchange.cu")],
+           *[os.path.join(csrc, n) for n in ("signsgd.cu", "variants.cu", "stats.cu", "exchange.cu", "vote_staged.cu")],
            os.path.join(ROOT, "tests", "sanitizer_abi_driver.cpp"), "-o", exe]
     res = subprocess.run(cmd, capture_output=True, text=True, timeout=900)
     assert res.returncode == 0, res.stderr[-2000:]
