@@ -47,7 +47,8 @@ NCU_TRAFFIC = {
         # profiles/worker_vote_apply_kernels_d2p25_M16_ncu_full.md
         "worker_pack_kernel:M16": {"bytes_per_param": (4.294976e9 + 2.164599e9) / 33554432, "d": 33554432},
         "vote_kernel:M16": {"bytes_per_param": (67.119e6 + 0.816e6) / 33554432, "d": 33554432},
-        # (apply_kernel: in the reduced capture x is partly L2-resident, so its traffic does not scale with d)
+        "apply_kernel:M16": {"bytes_per_param": None, "d": 33554432,
+                             "why": "in the reduced ncu capture x is partly L2-resident, so its traffic does not scale with d"},
         # profiles/fused_step_kernel_resnet50_M7_ncu_full.md (captured at full size)
         "fused_step_kernel:M7": {"bytes_per_param": (1.533629e9 + 793.557504e6) / 25557056, "d": 25557056},
     },
@@ -81,6 +82,8 @@ def ncu_traffic(kernel: str, M: int, d: int):
     rec = NCU_TRAFFIC["per_param"].get("%s:M%d" % (kernel, M))
     if rec is None:
         return None, "no ncu capture of this kernel at this M"
+    if rec["bytes_per_param"] is None:
+        return None, rec["why"]
     if rec["d"] == d:
         return rec["bytes_per_param"] * d, "ncu capture at this size"
     return rec["bytes_per_param"] * d, "scaled by d from the ncu capture at d = %d" % rec["d"]
