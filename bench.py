@@ -39,16 +39,17 @@ NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per parameter of one launch, from the ncu
-# captures summarised in profiles/ (taken at a reduced d with the same M and kernels; the path is
-# elementwise, so traffic grows in proportion to d).  Valid only while the kernel sources are unchanged.
+# captures summarised in profiles/.  At the captured size the figure is the capture's own; at another d
+# with the same M it is scaled (the path is elementwise, so traffic grows in proportion to d as long as
+# the operands exceed L2).  Valid only while the kernel sources are unchanged.
 NCU_TRAFFIC = {
     "source_sha256": "af53dee7a9e6e3f6abcc1924996a3536224d2db4a641aadf25a3ce8723d581fc",
     "per_param": {
-        # profiles/worker_vote_apply_kernels_d2p25_M16_ncu_full.md
-        "worker_pack_kernel:M16": {"bytes_per_param": (4.294976e9 + 2.164599e9) / 33554432, "d": 33554432},
-        "vote_kernel:M16": {"bytes_per_param": (67.119e6 + 0.816e6) / 33554432, "d": 33554432},
-        "apply_kernel:M16": {"bytes_per_param": None, "d": 33554432,
-                             "why": "in the reduced ncu capture x is partly L2-resident, so its traffic does not scale with d"},
+        # profiles/dram_bytes_worker_vote_apply_bertlarge_M16_full_size.md: a one-pass capture of the full-size
+        # default workload (d = 335,141,888)
+        "worker_pack_kernel:M16": {"bytes_per_param": (42900373760 + 22069851904) / 335141888, "d": 335141888},
+        "vote_kernel:M16": {"bytes_per_param": (670295040 + 36604672) / 335141888, "d": 335141888},
+        "apply_kernel:M16": {"bytes_per_param": (1382475008 + 1277894912) / 335141888, "d": 335141888},
         # profiles/fused_step_kernel_resnet50_M7_ncu_full.md (captured at full size)
         "fused_step_kernel:M7": {"bytes_per_param": (1.533629e9 + 793.557504e6) / 25557056, "d": 25557056},
     },
@@ -82,8 +83,6 @@ def ncu_traffic(kernel: str, M: int, d: int):
     rec = NCU_TRAFFIC["per_param"].get("%s:M%d" % (kernel, M))
     if rec is None:
         return None, "no ncu capture of this kernel at this M"
-    if rec["bytes_per_param"] is None:
-        return None, rec["why"]
     if rec["d"] == d:
         return rec["bytes_per_param"] * d, "ncu capture at this size"
     return rec["bytes_per_param"] * d, "scaled by d from the ncu capture at d = %d" % rec["d"]
