@@ -583,7 +583,7 @@ def test_abstention_shrinks_wrong_decisions_on_noisy_small_gradients():
 # ---------------------------------------------------------------- Section 3: density and Welford
 
 def test_density_of_dense_and_one_hot_vectors():
-    # "for a fully dense vector phi = 1 and for a fully sparse vector phi = 1/d"
+    # Sec. 3 gives the two end points of phi: 1 when every component has the same magnitude, 1/d for a one-hot vector
     d = 1000
     r = rng(81)
     dense = (3.0 * r.choice([-1.0, 1.0], d)).astype(np.float32)
