@@ -113,7 +113,9 @@ bool launch_scatter_u(const float* g, float* m, const PeerRows& dst, size_t P, s
   const unsigned long long tiles = (d + TILE - 1) / TILE;
   if (tiles > kMaxGrid) return false;
   const float omb = 1.0f - beta;
-  pack_scatter_kernel<MOMENTUM, UNROLL, !SPLIT><<<(unsigned)tiles, kThreads, 0, s>>>(g, m, dst, (unsigned)P, d, beta, omb);
+  // the same unused 36 KB shared-memory request as the worker kernel of the single-GPU step (carve-out hint)
+  const size_t smem = SPLIT ? 36 * 1024 : 0;
+  pack_scatter_kernel<MOMENTUM, UNROLL, !SPLIT><<<(unsigned)tiles, kThreads, smem, s>>>(g, m, dst, (unsigned)P, d, beta, omb);
   if constexpr (SPLIT) {
     if (d % (128 * UNROLL) != 0)
       pack_scatter_tail_kernel<MOMENTUM, UNROLL><<<1, 32, 0, s>>>(g, m, dst, (unsigned)P, d, beta, omb);
