@@ -11,7 +11,7 @@
 //
 // Peer memory is only ever WRITTEN here, with plain 32-bit stores; the vote kernel
 // later reads the rank's own copy of the rows from its own HBM.  No loads from
-// peer memory, no multicast, no waits inside the kernel: ordering between ranks
+// peer memory, no cluster-wide copies, no waits inside the kernel: ordering between ranks
 // (all rows have landed before a rank votes; a rank has finished voting before
 // its rows are overwritten) is the caller's, on the host or by a barrier kernel
 // between this launch and the vote.

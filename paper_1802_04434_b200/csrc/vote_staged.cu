@@ -10,7 +10,7 @@
 // One CTA owns a tile of 1024 consecutive words (one 128-bit chunk per thread) and
 // walks the M rows in groups of 8.  For every group one elected thread arms an
 // mbarrier with the group's byte count and issues one bulk copy per row (4 KB,
-// global -> shared, non-multicast, completion counted on the mbarrier); the groups
+// global -> this CTA's shared memory only, completion counted on the mbarrier); the groups
 // are double-buffered, so the copies of group i + 1 fly while group i is counted.
 // All threads wait for the group's mbarrier phase, read their 128-bit chunk of
 // each row from shared memory and fold it into the same bit-sliced carry-save
