@@ -172,6 +172,33 @@ def run_variants(d: int, M: int, reps: int, dev) -> list:
     return rows
 
 
+def run_yardsticks(log2n: int, reps: int, dev) -> list:
+    """Plain streaming library kernels over 2^log2n floats, as yardsticks for what this board's HBM gives to
+    each read : write mix (nothing here is part of the step): (name, us, GB/s) rows."""
+    n = 1 << log2n
+    a, b = torch.randn(n, device=dev), torch.randn(n, device=dev)
+    c = torch.empty(n, device=dev)
+    g = torch.randn(4, n // 4, device=dev)
+    m = torch.zeros(4, n // 4, device=dev)
+    bits = torch.zeros(4, n // 128, dtype=torch.int32, device=dev)
+    cases = [
+        ("torch add c <- a + b (2 reads : 1 write)", lambda: torch.add(a, b, out=c), 12 * n),
+        ("torch add_ a <- a + b in place (2 : 1)", lambda: a.add_(b, alpha=1e-6), 12 * n),
+        ("torch lerp_ a <- a + w (b - a) in place (2 : 1)", lambda: a.lerp_(b, 0.1), 12 * n),
+        ("ssgd_signum_momentum_pack, M = 4 (2 : 1 + 1/8)", lambda: B.signum_momentum_pack(g, m, 4, n // 4, n // 4, 0.9, bits, n // 128), 12.125 * n),
+        ("torch mul_ a <- 0.999 a in place (1 : 1)", lambda: a.mul_(0.999), 8 * n),
+        ("ssgd_sign_apply (1 : 1 + 1/8)", lambda: B.sign_apply(a, bits.view(-1), n, 1e-7), 8.125 * n),
+        ("torch sum(a) (read only)", lambda: torch.sum(a), 4 * n),
+        ("ssgd_sign_pack, M = 4 (read only + 1/8)", lambda: B.sign_pack(g, 4, n // 4, n // 4, bits, n // 128), 4.125 * n),
+        ("torch fill_ (write only)", lambda: c.fill_(1.0), 4 * n),
+    ]
+    rows = []
+    for name, fn, nbytes in cases:
+        ms = time_launches(lambda s: fn(), 1, reps)
+        rows.append((name, ms * 1e3, nbytes / (ms * 1e-3) / 1e9))
+    return rows
+
+
 def main(argv=None):
     ap = argparse.ArgumentParser()
     ap.add_argument("--min-log2", type=int, default=10)
@@ -182,6 +209,8 @@ def main(argv=None):
     ap.add_argument("--plain", action="store_true",
                     help="issue every launch from the host instead of replaying a CUDA graph (times then include "
                          "the host's per-call cost; meant for runs under a profiler)")
+    ap.add_argument("--yardsticks", type=int, default=None, metavar="LOG2N",
+                    help="instead of the sweep, time plain streaming library kernels (and this library's) over 2^LOG2N floats")
     ap.add_argument("--variants", default=None, metavar="LOG2D,M",
                     help="instead of the sweep, time the calls beside the main path at d = 2^LOG2D with M workers")
     args = ap.parse_args(argv)
@@ -191,6 +220,11 @@ def main(argv=None):
     PLAIN_LAUNCHES = args.plain
     dev = torch.device("cuda", 0)
     B.lib()
+    if args.yardsticks is not None:
+        print("kernel\tus_per_launch\tGBps\tfrac_of_measured_peak")
+        for name, us, gbs in run_yardsticks(args.yardsticks, max(2, args.reps // 4), dev):
+            print("%s\t%.1f\t%.0f\t%.3f" % (name, us, gbs, gbs / peak_gbs()), flush=True)
+        return 0
     out = open(args.out, "w") if args.out else None
     header = "d\tM\tkernel\tus_per_launch\talgorithmic_GBps\tfrac_of_measured_peak\tcold"
     print(header)
