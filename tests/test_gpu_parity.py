@@ -347,6 +347,35 @@ def test_config2_resnet50_layout():
     assert end < cfg.d and votes[end:].all()
 
 
+def test_config2_per_tensor_slices_of_the_wire_words():
+    """Every tensor of the bucketed vector starts on a word boundary, so a tensor's own sign words are a plain
+    slice of the row: packing one tensor alone (a call on that slice) gives exactly the words the whole-vector
+    call wrote at the tensor's word offset."""
+    cfg = wl.resnet50_signum()
+    M, d, ld, ldw = cfg.M, cfg.d, cfg.ld, cfg.ldw
+    gd = cfg.g(0, DEV)
+    bits = torch.zeros(M, ldw, dtype=torch.int32, device=DEV)
+    B.sign_pack(gd, M, d, ld, bits, ldw)
+    whole = u32(bits)
+    picks = [0, 1, 2, 57, 159, 160]                       # stem conv, two batch-norm vectors, a mid conv, fc weight, fc bias
+    for t in picks:
+        off, size = cfg.segments[t]
+        assert off % 32 == 0
+        W_t = oracle.words(size)
+        ldw_t = wl.round_up(W_t, 4)
+        ld_t = wl.round_up(size, 4)
+        g_t = torch.zeros(M, ld_t, device=DEV)
+        g_t[:, :size] = gd[:, off:off + size]
+        b_t = torch.zeros(M, ldw_t, dtype=torch.int32, device=DEV)
+        B.sign_pack(g_t, M, size, ld_t, b_t, ldw_t)
+        mine = whole[:, off // 32:off // 32 + W_t].copy()
+        if size % 32:                                     # the slice's last word also holds the pad elements (g = 0: bit 1)
+            mine[:, -1] &= np.uint32((1 << (size % 32)) - 1)
+        assert np.array_equal(u32(b_t)[:, :W_t], mine), "tensor %d" % t
+        ref = oracle.sign_pack(np.ascontiguousarray(f32(g_t)).reshape(-1), M, size, ld=ld_t, ldw=ldw_t).reshape(M, ldw_t)
+        assert np.array_equal(u32(b_t)[:, :W_t], ref[:, :W_t])
+
+
 def test_config3_ties_and_zeros():
     cfg = wl.tie_zero_stress()
     g, v_ref = run_config_full(cfg)
