@@ -43,19 +43,19 @@ FALLBACK_HBM_GBS = 6650.0
 # with the same M it is scaled (the path is elementwise, so traffic grows in proportion to d as long as
 # the operands exceed L2).  Valid only while the kernel sources are unchanged.
 NCU_TRAFFIC = {
-    "source_sha256": "af53dee7a9e6e3f6abcc1924996a3536224d2db4a641aadf25a3ce8723d581fc",
+    "source_sha256": "0f499230967ab8eddbaf6bf84031538c670786ae2d97361ca0c85e34a298775e",
     "per_param": {
         # profiles/dram_bytes_worker_vote_apply_bertlarge_M16_full_size.md: a one-pass capture of the full-size
         # default workload (d = 335,141,888)
-        "worker_pack_kernel:M16": {"bytes_per_param": (42900373760 + 22069851904) / 335141888, "d": 335141888},
-        "vote_kernel:M16": {"bytes_per_param": (670295040 + 36604672) / 335141888, "d": 335141888},
-        "apply_kernel:M16": {"bytes_per_param": (1382475008 + 1277894912) / 335141888, "d": 335141888},
+        "worker_pack_kernel:M16": {"bytes_per_param": (42898816000 + 22068206848) / 335141888, "d": 335141888},
+        "vote_kernel:M16": {"bytes_per_param": (670328832 + 36226816) / 335141888, "d": 335141888},
+        "apply_kernel:M16": {"bytes_per_param": (1382506496 + 1277509888) / 335141888, "d": 335141888},
         # profiles/fused_step_kernel_resnet50_M7_ncu_full.md (captured at full size)
-        "fused_step_kernel:M7": {"bytes_per_param": (1.533629e9 + 793.557504e6) / 25557056, "d": 25557056},
+        "fused_step_kernel:M7": {"bytes_per_param": (1.533635e9 + 792.759296e6) / 25557056, "d": 25557056},
     },
 }
 
-KERNEL_SOURCES = ("signsgd.cu", "device_common.cuh", "host_common.h")
+KERNEL_SOURCES = ("signsgd.cu", "device_common.cuh", "host_common.h", "vote_launch.h")
 
 
 def kernel_source_digest():

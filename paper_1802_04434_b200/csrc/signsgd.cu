@@ -19,6 +19,7 @@
 // no reuse for shared memory to serve, only an extra hop.
 
 #include "host_common.h"
+#include "vote_launch.h"
 
 namespace {
 
@@ -341,6 +342,11 @@ fused_step_kernel(const float* __restrict__ g, float* __restrict__ m, float* __r
 
 // ---------------------------------------------------------------------------
 // host side
+
+ssgd_status launch_vote(const uint32_t* bits, size_t M, size_t d, size_t ldw, uint32_t* vote,
+                        cudaStream_t s) {
+  return launch_vote_any<false>(bits, M, d, ldw, vote, 0, s);
+}
 
 constexpr size_t kWorkerSharedHint = 36 * 1024;   // below the 48 KB that need no opt-in
 

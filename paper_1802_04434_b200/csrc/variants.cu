@@ -7,6 +7,7 @@
 // See include/signsgd.h for the contract of each call.
 
 #include "host_common.h"
+#include "vote_launch.h"
 
 namespace {
 
