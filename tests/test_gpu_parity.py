@@ -296,6 +296,25 @@ def test_warmup_large_odd_d(d, M):
     assert_same_f32(f32(md).reshape(-1), m_ref, "m")
 
 
+@pytest.mark.parametrize("M,d", [(100, 40_001), (1000, 5_000), (1024, 4_097)])
+def test_whole_step_many_workers(M, d):
+    # grid rows up to the worker limit, ten and eleven counter planes in the vote
+    ld, W = wl.round_up(d, 4), oracle.words(d)
+    ldw = wl.round_up(W, 4)
+    g, m, x = rand_inputs(M, d, ld, seed=M + d)
+    gd, md, xd = (torch.from_numpy(a).to(DEV) for a in (g, m, x))
+    bits = torch.zeros(M, ldw, dtype=torch.int32, device=DEV)
+    vote = torch.zeros(W, dtype=torch.int32, device=DEV)
+    B.signsgd_step(xd, gd, md, M, d, ld, 0.9, 1e-3, bits, ldw, vote)
+    m_ref, x_ref = m.copy().reshape(-1), x.copy()
+    b_ref, v_ref = oracle.signsgd_step(x_ref, g.reshape(-1), m_ref, M, d, 0.9, 1e-3, ld=ld, ldw=ldw)
+    assert np.array_equal(u32(bits).reshape(-1), b_ref) and np.array_equal(u32(vote), v_ref)
+    assert_same_f32(f32(xd), x_ref, "x")
+    assert_same_f32(f32(md).reshape(-1), m_ref, "m")
+    with pytest.raises(B.SignSGDError):
+        B.signsgd_step(xd, gd, md, 1025, 4, 4, 0.9, 1e-3, bits, 4, vote)       # beyond the worker limit
+
+
 def test_empty_input_launches_nothing():
     z = torch.zeros(4, dtype=torch.float32, device=DEV)
     b = torch.full((4,), CANARY_WORD, dtype=torch.int32, device=DEV)
