@@ -128,12 +128,9 @@ ssgd_status launch_scatter(const float* g, float* m, const PeerRows& dst, size_t
                            cudaStream_t s) {
   DeviceInfo di;
   if (!device_info(&di)) return SSGD_ERR_CUDA;
-  bool ok;
-  switch (pick_unroll(d, 1, di.sms, 4)) {
-    case 4: ok = launch_scatter_u<MOMENTUM, 4>(g, m, dst, P, d, beta, s); break;
-    case 2: ok = launch_scatter_u<MOMENTUM, 2>(g, m, dst, P, d, beta, s); break;
-    default: ok = launch_scatter_u<MOMENTUM, 1>(g, m, dst, P, d, beta, s); break;
-  }
+  // tile sizes as for the worker kernel with a momentum (one row)
+  const bool ok = worker_unroll(d, 1, di.sms, true) == 4 ? launch_scatter_u<MOMENTUM, 4>(g, m, dst, P, d, beta, s)
+                                                         : launch_scatter_u<MOMENTUM, 1>(g, m, dst, P, d, beta, s);
   return ok ? launch_status() : SSGD_ERR_SIZE;
 }
 

@@ -56,17 +56,34 @@ ssgd_status launch_status() { return cudaGetLastError() == cudaSuccess ? SSGD_OK
 constexpr unsigned long long kMaxGrid = 0x7FFFFFFFull;
 unsigned grid_for(unsigned long long ctas) { return (unsigned)(ctas < kMaxGrid ? ctas : kMaxGrid); }
 
-// Elements per thread: 4 * unroll.  Large inputs take the largest unroll allowed
-// (eight 128-bit loads in flight per thread in the worker step); smaller ones
-// shrink the tile so that the launch still fills the machine with a few CTAs per SM.
-int pick_unroll(unsigned long long elements_per_row, unsigned long long rows, int sms, int max_unroll = 4) {
-  const unsigned long long want = 8ull * sms;                  // CTAs
-  for (int u = max_unroll; u > 1; u /= 2) {
-    const unsigned long long tile = (unsigned long long)kThreads * 4 * u;
-    if (((elements_per_row + tile - 1) / tile) * rows >= want) return u;
-  }
-  return 1;
+// Tile choice.  A thread handles 4 * unroll elements of one row, a CTA a tile of kThreads * 4 * unroll.
+// Large tiles give each thread more independent loads in flight and suit long streams; small tiles give a
+// short launch more CTAs to spread over the SMs.  The crossovers below were measured on B200 (148 SMs) by
+// forcing every tile size over d = 2^14 .. 2^27 and M = 1 .. 16, and are stated in tiles per SM.
+inline unsigned long long tile_count(unsigned long long elements_per_row, unsigned long long rows, int unroll) {
+  const unsigned long long tile = (unsigned long long)kThreads * 4 * unroll;
+  return ((elements_per_row + tile - 1) / tile) * rows;
 }
+
+// Worker kernel.  With a momentum: the interior-only 4096-element tiles win from about 64 Mi elements on
+// (2-4 % over 1024-element tiles), below that the 1024-element tiles win by 1-5 %; 2048 is never best.
+// Sign-only (one array): 8192-element tiles from about 32 Mi elements, 2048 from about 1.5 Mi, else 1024.
+inline int worker_unroll(unsigned long long d, unsigned long long rows, int sms, bool momentum) {
+  if (momentum) return tile_count(d, rows, 4) >= 112ull * sms ? 4 : 1;
+  if (tile_count(d, rows, 8) >= 24ull * sms) return 8;
+  return tile_count(d, rows, 2) >= 5ull * sms ? 2 : 1;
+}
+
+// Fused step kernel (a CTA walks all rows of its columns): the larger tile as soon as it still gives
+// three CTAs per SM (17-40 % faster than the next smaller tile at d = 2^20 .. 2^21, equal from 2^22 on).
+inline int fused_unroll(unsigned long long d, int sms, bool momentum) {
+  if (!momentum && tile_count(d, 1, 4) >= 3ull * sms) return 4;
+  return tile_count(d, 1, 2) >= 3ull * sms ? 2 : 1;
+}
+
+// Apply kernel: interior-only 2048-element tiles once they fill the machine 8 CTAs deep (no measurable
+// difference between the tile sizes below that).
+inline int apply_unroll(unsigned long long d, int sms) { return tile_count(d, 1, 2) >= 8ull * sms ? 2 : 1; }
 
 unsigned vote_planes(size_t M) {
   unsigned L = 0;

@@ -377,13 +377,17 @@ ssgd_status launch_worker(const float* g, float* m, size_t M, size_t d, size_t l
                           uint32_t* bits, size_t ldw, cudaStream_t s) {
   DeviceInfo di;
   if (!device_info(&di)) return SSGD_ERR_CUDA;
-  // without a momentum there is one array to load: twice the elements per thread keep as many loads in flight
   bool ok;
-  switch (pick_unroll(d, M, di.sms, MODE == kSignSGD ? 8 : 4)) {
-    case 8: ok = launch_worker_u<kSignSGD, 8>(g, m, M, d, ld, beta, bits, ldw, s); break;
-    case 4: ok = launch_worker_u<MODE, 4>(g, m, M, d, ld, beta, bits, ldw, s); break;
-    case 2: ok = launch_worker_u<MODE, 2>(g, m, M, d, ld, beta, bits, ldw, s); break;
-    default: ok = launch_worker_u<MODE, 1>(g, m, M, d, ld, beta, bits, ldw, s); break;
+  if constexpr (MODE == kSignSGD) {
+    // one array to load: twice the elements per thread keep as many loads in flight
+    switch (worker_unroll(d, M, di.sms, false)) {
+      case 8: ok = launch_worker_u<kSignSGD, 8>(g, m, M, d, ld, beta, bits, ldw, s); break;
+      case 2: ok = launch_worker_u<kSignSGD, 2>(g, m, M, d, ld, beta, bits, ldw, s); break;
+      default: ok = launch_worker_u<kSignSGD, 1>(g, m, M, d, ld, beta, bits, ldw, s); break;
+    }
+  } else {
+    ok = worker_unroll(d, M, di.sms, true) == 4 ? launch_worker_u<MODE, 4>(g, m, M, d, ld, beta, bits, ldw, s)
+                                                : launch_worker_u<MODE, 1>(g, m, M, d, ld, beta, bits, ldw, s);
   }
   return ok ? launch_status() : SSGD_ERR_SIZE;
 }
@@ -405,8 +409,8 @@ ssgd_status launch_apply(float* x, const uint32_t* vote, size_t d, float delta, 
   if (!device_info(&di)) return SSGD_ERR_CUDA;
   // 2048-element tiles, interior-only, once they fill the machine 8 CTAs deep; below that the smallest
   // tile with the guarded path inline (one launch)
-  const bool ok = pick_unroll(d, 1, di.sms, 2) == 2 ? launch_apply_u<2, true>(x, vote, d, delta, s)
-                                                   : launch_apply_u<1, false>(x, vote, d, delta, s);
+  const bool ok = apply_unroll(d, di.sms) == 2 ? launch_apply_u<2, true>(x, vote, d, delta, s)
+                                               : launch_apply_u<1, false>(x, vote, d, delta, s);
   return ok ? launch_status() : SSGD_ERR_SIZE;
 }
 
@@ -450,10 +454,8 @@ ssgd_status launch_fused(const StepArgs& a, cudaStream_t s, bool* launched) {
   DeviceInfo di;
   if (!device_info(&di)) return SSGD_ERR_CUDA;
   // Elements per thread and row: 8 with a momentum (two arrays to load: four 128-bit loads in flight),
-  // 16 without (one array), less for short vectors so that the launch still fills the machine.
-  const int want = MODE == kSignSGD ? 4 : 2;
-  const int fit = pick_unroll(a.d, 1, di.sms);
-  const int unroll = fit < want ? fit : want;
+  // 16 without (one array), less for short vectors (see fused_unroll).
+  const int unroll = fused_unroll(a.d, di.sms, MODE != kSignSGD);
   const unsigned long long tile = (unsigned long long)kThreads * 4 * unroll;
   if ((a.d + tile - 1) / tile > kMaxGrid) return SSGD_OK;
   bool ok;

@@ -211,8 +211,8 @@ def test_whole_step_small(M):
 
 
 # Odd vector lengths large enough that the launchers pick their largest tiles (16 and 32 elements per
-# thread), so that those instantiations meet a ragged last tile, a last word with pad bits, and rows
-# whose stride exceeds d.
+# thread: from about 64 Mi elements with a momentum, 32 Mi without), so that those instantiations meet a
+# ragged last tile, a last word with pad bits, and rows whose stride exceeds d.
 BIG_ODD_D = [5_000_003, (1 << 23) + 4099]
 
 
@@ -234,7 +234,7 @@ def check_rows(bits, ref, M, ldw, W, what):
 
 
 @pytest.mark.parametrize("d", BIG_ODD_D)
-@pytest.mark.parametrize("M", [1, 3])
+@pytest.mark.parametrize("M", [1, 3, 7])
 def test_sign_pack_large_odd_d(d, M):
     ld, W = wl.round_up(d, 4) + 8, oracle.words(d)
     ldw = wl.round_up(W, 4) + 4
@@ -245,7 +245,7 @@ def test_sign_pack_large_odd_d(d, M):
 
 
 @pytest.mark.parametrize("d", BIG_ODD_D)
-@pytest.mark.parametrize("M,beta,with_m", [(1, 0.0, False), (8, 0.0, False), (16, 0.9, True), (5, 0.9, True)])
+@pytest.mark.parametrize("M,beta,with_m", [(1, 0.0, False), (8, 0.0, False), (16, 0.9, True), (5, 0.9, True), (12, 0.0, False)])
 def test_whole_step_large_odd_d(d, M, beta, with_m):
     ld, W = wl.round_up(d, 4) + 8, oracle.words(d)
     ldw = wl.round_up(W, 4) + 4

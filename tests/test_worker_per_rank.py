@@ -184,7 +184,7 @@ def test_emulated_ranks_with_the_fused_pack_and_scatter_kernel(world, d, momentu
 
 
 @pytest.mark.gpu
-@pytest.mark.parametrize("d", [1, 33, 4097, 100_003, 5_000_003])
+@pytest.mark.parametrize("d", [1, 33, 4097, 100_003, 5_000_003, 70_000_003])
 def test_pack_scatter_kernel_matches_oracle_and_touches_nothing_else(d):
     from paper_1802_04434_b200 import binding as B
     dev = torch.device("cuda", 0)
