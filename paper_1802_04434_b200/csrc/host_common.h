@@ -52,6 +52,24 @@ inline bool beta_ok(float beta) { return beta >= 0.0f && beta < 1.0f; }  // fals
 
 ssgd_status launch_status() { return cudaGetLastError() == cudaSuccess ? SSGD_OK : SSGD_ERR_CUDA; }
 
+// Kernel launch with or without the programmatic-serialization attribute (see pdl_wait in
+// device_common.cuh).  Only kernels that begin with pdl_wait() may be launched with it.
+template <typename... KArgs, typename... Args>
+void launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, bool pdl,
+                   Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = pdl ? 1 : 0;
+  (void)cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);   // errors are read by launch_status()
+}
+
 // One tile per CTA; the kernels keep a grid-stride loop for grids beyond the limit.
 constexpr unsigned long long kMaxGrid = 0x7FFFFFFFull;
 unsigned grid_for(unsigned long long ctas) { return (unsigned)(ctas < kMaxGrid ? ctas : kMaxGrid); }
@@ -84,6 +102,19 @@ inline int fused_unroll(unsigned long long d, int sms, bool momentum) {
 // Apply kernel: interior-only 2048-element tiles once they fill the machine 8 CTAs deep (no measurable
 // difference between the tile sizes below that).
 inline int apply_unroll(unsigned long long d, int sms) { return tile_count(d, 1, 2) >= 8ull * sms ? 2 : 1; }
+
+// Vote kernel: the remaining rows after the batches of eight come as one guarded batch (see vote_kernel)
+// with four to six planes (M = 8 .. 127: 5-20 % faster at every size measured), and with three planes
+// (M = 4 .. 7) while the launch is at most four CTAs per SM deep (beyond that its 56 registers cost
+// more than the round trips save).  With more planes the kernel makes eight and more round trips
+// anyway and the guarded form would go from 64 to 72-80 registers; with fewer it has nothing to save.
+// Crossovers measured on B200.
+constexpr int kGuardedMinPlanes = 3;
+constexpr int kGuardedMaxPlanes = 6;
+inline bool vote_guarded(unsigned planes, unsigned long long ctas, int sms) {
+  if (planes == 3) return ctas <= 4ull * sms;
+  return planes > 3 && planes <= (unsigned)kGuardedMaxPlanes;
+}
 
 unsigned vote_planes(size_t M) {
   unsigned L = 0;

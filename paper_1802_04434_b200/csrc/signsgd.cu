@@ -76,6 +76,7 @@ worker_pack_kernel(const float* __restrict__ g, float* __restrict__ m,
   constexpr bool SIGN_OF_G = MODE != kSignum;
   constexpr unsigned long long TILE = (unsigned long long)kThreads * 4 * UNROLL;
   constexpr unsigned SPAN = 128 * UNROLL;
+  pdl_launch_dependents();   // in a step the vote kernel may be brought in while this grid drains
   const unsigned lane = threadIdx.x & 31u;
   const unsigned warp = threadIdx.x >> 5;
   const unsigned long long row = blockIdx.y;
@@ -157,6 +158,7 @@ __device__ __forceinline__ void apply_ragged_span(float* __restrict__ x, const u
 template <int UNROLL, bool RAGGED>
 __global__ void __launch_bounds__(kThreads, 1)
 apply_kernel(float* __restrict__ x, const uint32_t* __restrict__ vote, unsigned long long d, float delta) {
+  pdl_wait();   // the vote may come from the kernel before this one on the stream
   constexpr unsigned long long TILE = (unsigned long long)kThreads * 4 * UNROLL;
   constexpr unsigned SPAN = 128 * UNROLL;
   const unsigned lane = threadIdx.x & 31u;
@@ -344,8 +346,8 @@ fused_step_kernel(const float* __restrict__ g, float* __restrict__ m, float* __r
 // host side
 
 ssgd_status launch_vote(const uint32_t* bits, size_t M, size_t d, size_t ldw, uint32_t* vote,
-                        cudaStream_t s) {
-  return launch_vote_any<false>(bits, M, d, ldw, vote, 0, s);
+                        cudaStream_t s, bool pdl = false) {
+  return launch_vote_any<false>(bits, M, d, ldw, vote, 0, s, pdl);
 }
 
 constexpr size_t kWorkerSharedHint = 36 * 1024;   // below the 48 KB that need no opt-in
@@ -393,24 +395,26 @@ ssgd_status launch_worker(const float* g, float* m, size_t M, size_t d, size_t l
 }
 
 template <int UNROLL, bool SPLIT>
-bool launch_apply_u(float* x, const uint32_t* vote, size_t d, float delta, cudaStream_t s) {
+bool launch_apply_u(float* x, const uint32_t* vote, size_t d, float delta, cudaStream_t s, bool pdl) {
   constexpr unsigned long long TILE = (unsigned long long)kThreads * 4 * UNROLL;
   const unsigned long long tiles = (d + TILE - 1) / TILE;
   if (tiles > kMaxGrid) return false;     // beyond any device's memory
-  apply_kernel<UNROLL, !SPLIT><<<(unsigned)tiles, kThreads, 0, s>>>(x, vote, d, delta);
+  launch_kernel(apply_kernel<UNROLL, !SPLIT>, (unsigned)tiles, kThreads, 0, s, pdl, x, vote,
+                (unsigned long long)d, delta);
   if constexpr (SPLIT) {
     if (d % (128 * UNROLL) != 0) apply_tail_kernel<UNROLL><<<1, 32, 0, s>>>(x, vote, d, delta);
   }
   return true;
 }
 
-ssgd_status launch_apply(float* x, const uint32_t* vote, size_t d, float delta, cudaStream_t s) {
+ssgd_status launch_apply(float* x, const uint32_t* vote, size_t d, float delta, cudaStream_t s,
+                         bool pdl = false) {
   DeviceInfo di;
   if (!device_info(&di)) return SSGD_ERR_CUDA;
   // 2048-element tiles, interior-only, once they fill the machine 8 CTAs deep; below that the smallest
   // tile with the guarded path inline (one launch)
-  const bool ok = apply_unroll(d, di.sms) == 2 ? launch_apply_u<2, true>(x, vote, d, delta, s)
-                                               : launch_apply_u<1, false>(x, vote, d, delta, s);
+  const bool ok = apply_unroll(d, di.sms) == 2 ? launch_apply_u<2, true>(x, vote, d, delta, s, pdl)
+                                               : launch_apply_u<1, false>(x, vote, d, delta, s, pdl);
   return ok ? launch_status() : SSGD_ERR_SIZE;
 }
 
@@ -476,9 +480,11 @@ ssgd_status run_step(const StepArgs& a, cudaStream_t s) {
   if (st != SSGD_OK || launched) return st;
   st = launch_worker<MODE>(a.g, a.m, a.M, a.d, a.ld, a.beta, a.bits, a.ldw, s);
   if (st != SSGD_OK) return st;
-  st = launch_vote(a.bits, a.M, a.d, a.ldw, a.vote, s);
+  // vote and apply follow this library's own kernels on the stream: programmatic dependent launch lets
+  // each be brought onto the SMs while its predecessor drains (both begin with pdl_wait())
+  st = launch_vote(a.bits, a.M, a.d, a.ldw, a.vote, s, true);
   if (st != SSGD_OK) return st;
-  return launch_apply(a.x, a.vote, a.d, a.delta, s);
+  return launch_apply(a.x, a.vote, a.d, a.delta, s, true);
 }
 
 // argument checks shared by the entry points -------------------------------

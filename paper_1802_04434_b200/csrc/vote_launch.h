@@ -9,9 +9,18 @@ namespace {
 
 template <int NP, bool COUNTS>
 void launch_vote_np(const uint32_t* bits, size_t M, size_t d, size_t W, size_t ldw, uint32_t* out,
-                    size_t ldc, unsigned grid, cudaStream_t s) {
+                    size_t ldc, unsigned grid, bool guarded, bool pdl, cudaStream_t s) {
   const unsigned start = COUNTS ? 0u : vote_start_value(M, NP);
-  vote_kernel<NP, COUNTS><<<grid, kThreads, 0, s>>>(bits, (unsigned)M, d, W, ldw, out, ldc, start);
+  const unsigned long long d64 = d, W64 = W, ldw64 = ldw, ldc64 = ldc;
+  if constexpr (NP >= kGuardedMinPlanes && NP <= kGuardedMaxPlanes) {   // the only ones vote_guarded() picks
+    if (guarded) {
+      launch_kernel(vote_kernel<NP, COUNTS, true>, grid, kThreads, 0, s, pdl, bits, (unsigned)M, d64, W64, ldw64,
+                    out, ldc64, start);
+      return;
+    }
+  }
+  launch_kernel(vote_kernel<NP, COUNTS, false>, grid, kThreads, 0, s, pdl, bits, (unsigned)M, d64, W64, ldw64,
+                out, ldc64, start);
 }
 
 // planes that hold a count in 0..M: the bit length of M
@@ -21,24 +30,25 @@ unsigned count_planes(size_t M) {
   return n;
 }
 
+// pdl: launch with the programmatic-serialization attribute (the step entry points, where the kernel
+// before this one on the stream is this library's own).
 template <bool COUNTS>
 ssgd_status launch_vote_any(const uint32_t* bits, size_t M, size_t d, size_t ldw, uint32_t* out,
-                            size_t ldc, cudaStream_t s) {
+                            size_t ldc, cudaStream_t s, bool pdl = false) {
+  DeviceInfo di;
+  if (!device_info(&di)) return SSGD_ERR_CUDA;
   const size_t W = ssgd_words(d);
   const unsigned long long chunks = (W + 3) / 4;
-  const unsigned grid = grid_for((chunks + kThreads - 1) / kThreads);
-  switch (COUNTS ? count_planes(M) : vote_planes(M)) {
-    case 1: launch_vote_np<1, COUNTS>(bits, M, d, W, ldw, out, ldc, grid, s); break;
-    case 2: launch_vote_np<2, COUNTS>(bits, M, d, W, ldw, out, ldc, grid, s); break;
-    case 3: launch_vote_np<3, COUNTS>(bits, M, d, W, ldw, out, ldc, grid, s); break;
-    case 4: launch_vote_np<4, COUNTS>(bits, M, d, W, ldw, out, ldc, grid, s); break;
-    case 5: launch_vote_np<5, COUNTS>(bits, M, d, W, ldw, out, ldc, grid, s); break;
-    case 6: launch_vote_np<6, COUNTS>(bits, M, d, W, ldw, out, ldc, grid, s); break;
-    case 7: launch_vote_np<7, COUNTS>(bits, M, d, W, ldw, out, ldc, grid, s); break;
-    case 8: launch_vote_np<8, COUNTS>(bits, M, d, W, ldw, out, ldc, grid, s); break;
-    case 9: launch_vote_np<9, COUNTS>(bits, M, d, W, ldw, out, ldc, grid, s); break;
-    case 10: launch_vote_np<10, COUNTS>(bits, M, d, W, ldw, out, ldc, grid, s); break;
-    case 11: launch_vote_np<11, COUNTS>(bits, M, d, W, ldw, out, ldc, grid, s); break;
+  const unsigned long long ctas = (chunks + kThreads - 1) / kThreads;
+  const unsigned grid = grid_for(ctas);
+  const unsigned planes = COUNTS ? count_planes(M) : vote_planes(M);
+  const bool g = vote_guarded(planes, ctas, di.sms);
+  switch (planes) {
+#define SSGD_VOTE_CASE(n) \
+  case n: launch_vote_np<n, COUNTS>(bits, M, d, W, ldw, out, ldc, grid, g, pdl, s); break;
+    SSGD_VOTE_CASE(1) SSGD_VOTE_CASE(2) SSGD_VOTE_CASE(3) SSGD_VOTE_CASE(4) SSGD_VOTE_CASE(5) SSGD_VOTE_CASE(6)
+    SSGD_VOTE_CASE(7) SSGD_VOTE_CASE(8) SSGD_VOTE_CASE(9) SSGD_VOTE_CASE(10) SSGD_VOTE_CASE(11)
+#undef SSGD_VOTE_CASE
     default: return SSGD_ERR_SIZE;
   }
   return launch_status();

@@ -113,6 +113,30 @@ def test_majority_vote_small(M):
         assert np.all(got[W:] == np.uint32(0xDEADBEEF))
 
 
+@pytest.mark.parametrize("M,d", [(5, (1 << 25) + 37), (7, (1 << 25) + 37), (7, 5_000_003), (4, 3_000_001),
+                                 (13, (1 << 24) + 4099), (31, 5_000_003), (63, 2_000_003), (64, 2_000_003),
+                                 (100, 1_000_003)])
+def test_majority_vote_long_vectors(M, d):
+    """Both forms of the vote kernel's tail (remaining rows in batches of 4, 2, 1, or as one guarded batch) on
+    launches many CTAs per SM deep and on shorter ones, with a ragged last word and garbage in the row padding."""
+    r = np.random.default_rng(M * 7919 + d % 1000)
+    W = oracle.words(d)
+    ldw = wl.round_up(W, 4) + 8
+    rows = r.integers(0, 2**32, size=(M, ldw), dtype=np.uint32)
+    # a band of elements where the count sits at the threshold: exactly ceil(M/2) and ceil(M/2) - 1 set bits
+    T = (M + 1) // 2
+    for j, ones in ((3, T), (W // 2, T - 1), (W - 2, T)):
+        rows[:, j] = 0
+        rows[:ones, j] = 0xFFFFFFFF
+    vote = torch.full((W + 4,), CANARY_WORD, dtype=torch.int32, device=DEV)
+    B.majority_vote(torch.from_numpy(rows.view(np.int32)).to(DEV), M, d, ldw, vote)
+    ref = oracle.majority_vote(rows.reshape(-1), M, d, ldw=ldw)
+    got = u32(vote)
+    assert got[3] == 0xFFFFFFFF and got[W // 2] == 0 and ref[3] == 0xFFFFFFFF and ref[W // 2] == 0
+    assert np.array_equal(got[:W], ref), "M=%d d=%d" % (M, d)
+    assert np.all(got[W:] == np.uint32(0xDEADBEEF))
+
+
 @pytest.mark.parametrize("M", [1, 2, 3, 7, 8, 9, 16, 17, 31, 33, 100, 1024])
 def test_majority_vote_staged_through_shared_memory(M):
     # the second kernel design (rows staged by bulk copies, 8 rows per mbarrier phase): same words
