@@ -383,12 +383,12 @@ def timed_block(step, K, stream, flush, torch):
 def per_kernel_pass(B, b, K, stream, flush, torch):
     """Second pass over the same buffers: CUDA-event pairs around every kernel of the step.
 
-    For M <= FUSED_MAX_WORKERS the step is one fused kernel; otherwise the three entry points the step
+    Where the step is one fused kernel it is timed as such; otherwise the three entry points the step
     entry point issues are called one by one so that events can sit between the kernels."""
     cfg = b.cfg
     M, d, ld, ldw = cfg.M, cfg.d, cfg.ld, cfg.ldw
     momentum = cfg.momentum_buffer
-    fused = M <= B.FUSED_MAX_WORKERS
+    fused = B.step_is_fused(M, d, momentum)
     ev = lambda: torch.cuda.Event(enable_timing=True)
     marks = []
     for _ in range(K):
@@ -465,7 +465,7 @@ def run_ours(args):
     b = Buffers(cfg, dev)
     stream = torch.cuda.current_stream()
     step = make_step(B, b, stream)
-    fused = M <= B.FUSED_MAX_WORKERS
+    fused = B.step_is_fused(M, d, momentum)
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev) if needs_l2_flush(cfg) else None
     K, Wm = args.steps, args.warmup
 

@@ -115,6 +115,15 @@ ssgd_status ssgd_signsgd_step(float* x, const float* g, float* m, size_t M,
                               uint32_t* bits_ws, size_t ldw, uint32_t* vote_ws,
                               void* stream);
 
+/* Launch shape of ssgd_signsgd_step on the current device (a query for
+ * measurement tools; the result of the step does not depend on it): 1 when the
+ * step for M workers and d parameters runs as ONE fused kernel (worker step of
+ * every row, vote and apply on a tile of columns: Algorithm 3 as a whole in one
+ * pass), 0 when it runs as the worker, vote and apply kernels one after another.
+ * momentum != 0 asks about the Signum step (m given), 0 about the sign-only step
+ * (m == NULL).  Returns 0 for M or d out of range or when no device is current.  */
+int ssgd_step_is_fused(size_t M, size_t d, int momentum);
+
 /* Theorem 3 (Signum): the warm-up length C(beta), the least positive integer C
  * with (C/2) beta^C <= 1 / ((1 - beta^2)(C + 1)) and beta^(C+1) <= 1/2; the
  * paper notes C(0.9) = 54.  Pure host arithmetic, no GPU work.  Returns 0 when

@@ -18,7 +18,6 @@ import torch
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libsignsgd_b200.so")
 MAX_WORKERS = 1024
-FUSED_MAX_WORKERS = 8      # ssgd_signsgd_step runs as one fused kernel up to this many workers
 
 _lib = None
 
@@ -48,6 +47,8 @@ def lib() -> ctypes.CDLL:
     L.ssgd_count_planes.argtypes = [sz]
     L.ssgd_warmup_steps.restype = sz
     L.ssgd_warmup_steps.argtypes = [f32]
+    L.ssgd_step_is_fused.restype = ci
+    L.ssgd_step_is_fused.argtypes = [sz, sz, ci]
     L.ssgd_status_str.restype = ctypes.c_char_p
     L.ssgd_status_str.argtypes = [ci]
     sigs = {
@@ -178,6 +179,12 @@ def signsgd_step(x: torch.Tensor, g: torch.Tensor, m: Optional[torch.Tensor], M:
         _ptr(x, torch.float32, "x"), _ptr(g, torch.float32, "g"), _ptr(m, torch.float32, "m"),
         M, d, ld, beta, delta, _ptr(bits_ws, WORD_DTYPE, "bits_ws"), ldw,
         _ptr(vote_ws, WORD_DTYPE, "vote_ws"), _stream(stream)), "ssgd_signsgd_step")
+
+
+def step_is_fused(M: int, d: int, momentum: bool) -> bool:
+    """Whether signsgd_step runs as one fused kernel for this problem on the current device (else worker,
+    vote and apply kernels); a query for measurement tools."""
+    return bool(lib().ssgd_step_is_fused(M, d, 1 if momentum else 0))
 
 
 def warmup_steps(beta: float) -> int:

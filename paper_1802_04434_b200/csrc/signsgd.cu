@@ -210,8 +210,10 @@ apply_tail_kernel(float* __restrict__ x, const uint32_t* __restrict__ vote, unsi
 // 2M + 1 concurrent row streams cost 1-5 % of DRAM efficiency against the worker
 // kernel's two, so the step entry point then uses the three kernels.
 
-constexpr int kFusedMaxWorkers = 8;   // rows walked by one CTA at most
-constexpr int kFusedMaxPlanes = 4;    // planes needed for M <= 8
+constexpr int kFusedMaxWorkers = 8;           // rows walked by one CTA at most, with a momentum
+constexpr int kFusedMaxWorkersSignOnly = 32;  // ... without one, on long vectors (see step_is_fused)
+constexpr int kFusedMaxPlanes = 4;            // planes needed for M <= 8
+constexpr int kFusedMaxPlanesSignOnly = 6;    // ... for M <= 32
 
 template <int MODE, int UNROLL, int NP>
 __device__ __forceinline__ void fused_row(const float* __restrict__ gr, float* __restrict__ mr,
@@ -445,23 +447,40 @@ bool launch_fused_mu(const StepArgs& a, cudaStream_t s) {
     case 3: launch_fused_mun<MODE, UNROLL, 3>(a, s); return true;
     case 4: launch_fused_mun<MODE, UNROLL, 4>(a, s); return true;
   }
+  if constexpr (MODE == kSignSGD && UNROLL == 4) {   // more than eight workers: sign-only, long vectors
+    switch (vote_planes(a.M)) {
+      case 5: launch_fused_mun<MODE, UNROLL, 5>(a, s); return true;
+      case 6: launch_fused_mun<MODE, UNROLL, 6>(a, s); return true;
+    }
+  }
   return false;
 }
 
-// Whether the step runs as the fused kernel: few workers, and a vector that fits
-// one grid of tiles.  Everything else takes the three kernels.
+// Whether the step runs as the fused kernel.  Up to eight workers: always (if the vector fits one grid
+// of tiles).  Nine to 32 workers: only without a momentum and on long vectors -- there the worker
+// kernel is a read-only stream and the x update rides along with it: measured on B200 at d >= 2^23 the
+// fused kernel is 8-13 % faster for M = 9 .. 12 and 2-3 % for M = 16 .. 31, while on shorter vectors,
+// and with a momentum at any size, the three kernels win by up to 5 %.
+template <int MODE>
+bool step_is_fused(size_t M, size_t d, int sms) {
+  static_assert(kFusedMaxWorkers / 2 < (1 << (kFusedMaxPlanes - 1)), "planes cover the fused worker limit");
+  static_assert(kFusedMaxWorkersSignOnly / 2 < (1 << (kFusedMaxPlanesSignOnly - 1)), "... and the sign-only one");
+  const int unroll = fused_unroll(d, sms, MODE != kSignSGD);
+  if (tile_count(d, 1, unroll) > kMaxGrid) return false;
+  if (M <= (size_t)kFusedMaxWorkers) return true;
+  return MODE == kSignSGD && M <= (size_t)kFusedMaxWorkersSignOnly && unroll == 4 &&
+         tile_count(d, 1, 4) >= 12ull * sms;
+}
+
 template <int MODE>
 ssgd_status launch_fused(const StepArgs& a, cudaStream_t s, bool* launched) {
-  static_assert(kFusedMaxWorkers / 2 < (1 << (kFusedMaxPlanes - 1)), "planes cover the fused worker limit");
   *launched = false;
-  if (a.M > (size_t)kFusedMaxWorkers) return SSGD_OK;
   DeviceInfo di;
   if (!device_info(&di)) return SSGD_ERR_CUDA;
+  if (!step_is_fused<MODE>(a.M, a.d, di.sms)) return SSGD_OK;
   // Elements per thread and row: 8 with a momentum (two arrays to load: four 128-bit loads in flight),
   // 16 without (one array), less for short vectors (see fused_unroll).
   const int unroll = fused_unroll(a.d, di.sms, MODE != kSignSGD);
-  const unsigned long long tile = (unsigned long long)kThreads * 4 * unroll;
-  if ((a.d + tile - 1) / tile > kMaxGrid) return SSGD_OK;
   bool ok;
   if (MODE == kSignSGD && unroll == 4) ok = launch_fused_mu<kSignSGD, 4>(a, s);
   else if (unroll == 2) ok = launch_fused_mu<MODE, 2>(a, s);
@@ -589,6 +608,12 @@ ssgd_status ssgd_signsgd_step(float* x, const float* g, float* m, size_t M, size
   const StepArgs a{g, m, x, bits_ws, vote_ws, M, d, ld, ldw, beta, delta};
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   return m ? run_step<kSignum>(a, s) : run_step<kSignSGD>(a, s);
+}
+
+int ssgd_step_is_fused(size_t M, size_t d, int momentum) {
+  DeviceInfo di;
+  if (M < 1 || M > SSGD_MAX_WORKERS || d == 0 || !device_info(&di)) return 0;
+  return (momentum ? step_is_fused<kSignum>(M, d, di.sms) : step_is_fused<kSignSGD>(M, d, di.sms)) ? 1 : 0;
 }
 
 size_t ssgd_warmup_steps(float beta) {

@@ -154,6 +154,11 @@ def run_variants(d: int, M: int, reps: int, dev) -> list:
         gbs = nbytes / (ms * 1e-3) / 1e9
         rows.append((d, M, name, ms * 1e3, gbs, gbs / peak_gbs(), int(nbytes >= 2 * L2_BYTES)))
 
+    # Algorithm 3 as printed (no momentum): one fused kernel up to 8 workers, and up to 32 on long vectors
+    sign_only_bytes = (4.125 * M + 8.125 + (0.0 if B.step_is_fused(M, d, False) else (M + 1) / 8.0)) * d
+    rec("signsgd_step_sign_only", time_launches(lambda s: B.signsgd_step(x, g, None, M, d, ld, 0.0, 1e-4, bits, ldw, vs),
+                                                1, reps), sign_only_bytes)
+    B.sign_pack(g, M, d, ld, bits, ldw)
     rec("signum_warmup_pack", time_launches(lambda s: B.signum_warmup_pack(g, m, M, d, ld, 0.9, bits, ldw), 1, reps),
         12.125 * M * d)
     rec("vote_counts", time_launches(lambda s: B.vote_counts(bits, M, d, ldw, counts, ldw), 1, reps),

@@ -153,6 +153,9 @@ def test_warmup_steps_is_host_arithmetic(L):
     assert L.ssgd_warmup_steps(0.9) == 54          # the value Theorem 3 prints for beta = 0.9
     assert L.ssgd_warmup_steps(0.0) == 1
     assert L.ssgd_warmup_steps(1.0) == 0 and L.ssgd_warmup_steps(float("nan")) == 0
+    # the launch-shape query answers 0 for sizes out of range (and, with no device, for everything)
+    assert L.ssgd_step_is_fused(0, 1000, 1) == 0 and L.ssgd_step_is_fused(1025, 1000, 0) == 0
+    assert L.ssgd_step_is_fused(3, 0, 1) == 0
     w = L.ssgd_signsgd_warmup_step
     assert w(A, A, None, 1, 64, 64, 0.9, 0.1, A, 4, A, None) == NULL     # m is required
     assert w(A, A, A, 1, 0, 0, 0.9, 0.1, A, 0, A, None) == OK

@@ -269,8 +269,14 @@ def test_sign_pack_large_odd_d(d, M):
 
 
 @pytest.mark.parametrize("d", BIG_ODD_D)
-@pytest.mark.parametrize("M,beta,with_m", [(1, 0.0, False), (8, 0.0, False), (16, 0.9, True), (5, 0.9, True), (12, 0.0, False)])
+@pytest.mark.parametrize("M,beta,with_m", [(1, 0.0, False), (8, 0.0, False), (16, 0.9, True), (5, 0.9, True), (12, 0.0, False),
+                                           (9, 0.0, False), (17, 0.0, False), (32, 0.0, False), (33, 0.0, False)])
 def test_whole_step_large_odd_d(d, M, beta, with_m):
+    # both launch shapes of the step occur here for the same M: without a momentum, 9 to 32 workers run as the
+    # one fused kernel on the longer vector and as worker + vote + apply kernels on the shorter one
+    if not with_m and 8 < M <= 32:
+        assert B.step_is_fused(M, d, False) == (d > 7_500_000)
+    assert B.step_is_fused(M, d, with_m) == (M <= 8 or (not with_m and M <= 32 and d > 7_500_000))
     ld, W = wl.round_up(d, 4) + 8, oracle.words(d)
     ldw = wl.round_up(W, 4) + 4
     g, m, x = big_inputs(M, d, ld, seed=d % 1000 + 7 * M, with_m=with_m)
