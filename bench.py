@@ -55,7 +55,7 @@ NCU_TRAFFIC = {
     },
 }
 
-KERNEL_SOURCES = ("signsgd.cu", "device_common.cuh", "host_common.h", "vote_launch.h")
+KERNEL_SOURCES = ("signsgd.cu", "device_common.cuh", "host_common.h", "vote_launch.h", "step_rows.cuh")
 
 
 def kernel_source_digest():
@@ -414,7 +414,7 @@ def per_kernel_pass(B, b, K, stream, flush, torch):
     n = len(marks[0]) - 1
     ms = [sum(e[i].elapsed_time(e[i + 1]) for e in marks) / K for i in range(n)]
     if fused:
-        names = [("fused_step_kernel", "ssgd_signsgd_step", fused_bpp(M, momentum))]
+        names = [(B.step_kernel_name(M, d, momentum), "ssgd_signsgd_step", fused_bpp(M, momentum))]
     else:
         names = [("worker_pack_kernel", "ssgd_signum_momentum_pack" if momentum else "ssgd_sign_pack",
                   worker_bpp(M, momentum)),

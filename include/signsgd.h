@@ -119,7 +119,9 @@ ssgd_status ssgd_signsgd_step(float* x, const float* g, float* m, size_t M,
  * measurement tools; the result of the step does not depend on it): 1 when the
  * step for M workers and d parameters runs as ONE fused kernel (worker step of
  * every row, vote and apply on a tile of columns: Algorithm 3 as a whole in one
- * pass), 0 when it runs as the worker, vote and apply kernels one after another.
+ * pass), 2 when it runs as the one-kernel form for short vectors (the rows of a
+ * tile handled by different warps at the same time), 0 when it runs as the
+ * worker, vote and apply kernels one after another.
  * momentum != 0 asks about the Signum step (m given), 0 about the sign-only step
  * (m == NULL).  Returns 0 for M or d out of range or when no device is current.  */
 int ssgd_step_is_fused(size_t M, size_t d, int momentum);

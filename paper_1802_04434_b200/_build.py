@@ -9,7 +9,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(_HERE)
 SOURCES = [os.path.join(_HERE, "csrc", n) for n in ("signsgd.cu", "variants.cu", "stats.cu", "exchange.cu", "vote_staged.cu")]
 HEADERS = [os.path.join(ROOT, "include", "signsgd.h")] + [
-    os.path.join(_HERE, "csrc", n) for n in ("device_common.cuh", "host_common.h", "vote_launch.h")]
+    os.path.join(_HERE, "csrc", n) for n in ("device_common.cuh", "host_common.h", "vote_launch.h", "step_rows.cuh")]
 LIB = os.path.join(_HERE, "libsignsgd_b200.so")
 
 NVCC_FLAGS = [

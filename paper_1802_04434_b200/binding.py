@@ -182,9 +182,14 @@ def signsgd_step(x: torch.Tensor, g: torch.Tensor, m: Optional[torch.Tensor], M:
 
 
 def step_is_fused(M: int, d: int, momentum: bool) -> bool:
-    """Whether signsgd_step runs as one fused kernel for this problem on the current device (else worker,
+    """Whether signsgd_step runs as one kernel for this problem on the current device (else worker,
     vote and apply kernels); a query for measurement tools."""
-    return bool(lib().ssgd_step_is_fused(M, d, 1 if momentum else 0))
+    return lib().ssgd_step_is_fused(M, d, 1 if momentum else 0) != 0
+
+
+def step_kernel_name(M: int, d: int, momentum: bool) -> str:
+    """Name of the kernel that is the whole step, or '' when the step is three kernels."""
+    return ("", "fused_step_kernel", "step_rows_kernel")[lib().ssgd_step_is_fused(M, d, 1 if momentum else 0)]
 
 
 def warmup_steps(beta: float) -> int:

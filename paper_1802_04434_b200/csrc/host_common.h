@@ -31,6 +31,17 @@ bool device_info(DeviceInfo* out) {
   return true;
 }
 
+// Arguments of one whole step (ssgd_signsgd_step and its warm-up form).
+struct StepArgs {
+  const float* g;
+  float* m;
+  float* x;
+  uint32_t* bits;
+  uint32_t* vote;
+  size_t M, d, ld, ldw;
+  float beta, delta;
+};
+
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 inline bool mul_overflows(size_t a, size_t b) { return b != 0 && a > SIZE_MAX / b; }

@@ -20,6 +20,7 @@
 
 #include "host_common.h"
 #include "vote_launch.h"
+#include "step_rows.cuh"
 
 namespace {
 
@@ -420,16 +421,6 @@ ssgd_status launch_apply(float* x, const uint32_t* vote, size_t d, float delta, 
   return ok ? launch_status() : SSGD_ERR_SIZE;
 }
 
-struct StepArgs {
-  const float* g;
-  float* m;
-  float* x;
-  uint32_t* bits;
-  uint32_t* vote;
-  size_t M, d, ld, ldw;
-  float beta, delta;
-};
-
 template <int MODE, int UNROLL, int NP>
 void launch_fused_mun(const StepArgs& a, cudaStream_t s) {
   constexpr unsigned long long TILE = (unsigned long long)kThreads * 4 * UNROLL;
@@ -490,10 +481,14 @@ ssgd_status launch_fused(const StepArgs& a, cudaStream_t s, bool* launched) {
   return launch_status();
 }
 
-// One whole step in the given worker mode: the fused kernel where it applies,
-// otherwise worker, vote and apply kernels on the same stream.
+// One whole step in the given worker mode: the row-parallel kernel for short vectors, the fused kernel
+// where it applies, otherwise worker, vote and apply kernels on the same stream.
 template <int MODE>
 ssgd_status run_step(const StepArgs& a, cudaStream_t s) {
+  DeviceInfo di;
+  if (!device_info(&di)) return SSGD_ERR_CUDA;
+  // short vectors: one launch whose warps work on different rows at once (step_rows.cuh)
+  if (step_uses_rows_kernel(a.M, a.d, di.sms, MODE != kSignSGD)) return launch_step_rows<MODE>(a, s);
   bool launched = false;
   ssgd_status st = launch_fused<MODE>(a, s, &launched);
   if (st != SSGD_OK || launched) return st;
@@ -613,6 +608,7 @@ ssgd_status ssgd_signsgd_step(float* x, const float* g, float* m, size_t M, size
 int ssgd_step_is_fused(size_t M, size_t d, int momentum) {
   DeviceInfo di;
   if (M < 1 || M > SSGD_MAX_WORKERS || d == 0 || !device_info(&di)) return 0;
+  if (step_uses_rows_kernel(M, d, di.sms, momentum != 0)) return 2;
   return (momentum ? step_is_fused<kSignum>(M, d, di.sms) : step_is_fused<kSignSGD>(M, d, di.sms)) ? 1 : 0;
 }
 

@@ -215,23 +215,36 @@ def test_sign_apply_small(d):
 
 @pytest.mark.parametrize("M", SMALL_M)
 def test_whole_step_small(M):
-    for d in (33, 1000, 4097, 70001):
+    # 33 .. 70001: one launch whose warps take different rows (2 <= M <= 32); 400003: past that kernel's range for
+    # every M, i.e. the fused kernel's smallest tile with a ragged span (M <= 8) or worker + vote + apply.
+    # Row strides longer than the rows, canaries behind every output.
+    for d in (33, 1000, 4097, 70001, 400_003):
         for beta, with_m in ((0.9, True), (0.0, True), (0.0, False)):
-            ld, W = wl.round_up(d, 4), oracle.words(d)
-            ldw = wl.round_up(W, 4)
-            g, m, x = rand_inputs(M, d, ld, seed=M * 77 + d)
+            shape = B.lib().ssgd_step_is_fused(M, d, 1 if with_m else 0)
+            if d < 400_003:
+                assert shape == (2 if 2 <= M <= 32 else (1 if M == 1 else 0)), (M, d, shape)
+            else:
+                assert shape == (1 if M <= 8 else 0), (M, d, shape)
+            ld, W = wl.round_up(d, 4) + 4, oracle.words(d)
+            ldw = wl.round_up(W, 4) + 4
+            g, m, x = rand_inputs(M, d, ld, seed=M * 77 + d, special=True)
+            x = np.concatenate([x, np.full(8, CANARY_F, dtype=np.float32)])
             gd, md, xd = (torch.from_numpy(a).to(DEV) for a in (g, m, x))
-            bits = torch.zeros(M, ldw, dtype=torch.int32, device=DEV)
-            vote = torch.zeros(W, dtype=torch.int32, device=DEV)
+            bits = torch.full((M, ldw), CANARY_WORD, dtype=torch.int32, device=DEV)
+            vote = torch.full((W + 4,), CANARY_WORD, dtype=torch.int32, device=DEV)
             B.signsgd_step(xd, gd, md if with_m else None, M, d, ld, beta, 1e-3, bits, ldw, vote)
-            m_ref, x_ref = m.copy().reshape(-1), x.copy()
+            m_ref, x_ref = m.copy().reshape(-1), x[:d].copy()
             b_ref, v_ref = oracle.signsgd_step(x_ref, g.reshape(-1), m_ref if with_m else None, M, d,
                                                beta, 1e-3, ld=ld, ldw=ldw)
-            assert np.array_equal(u32(bits).reshape(-1), b_ref)
-            assert np.array_equal(u32(vote), v_ref)
-            assert_same_f32(f32(xd), x_ref, "x")
+            what = "M=%d d=%d beta=%g m=%s" % (M, d, beta, with_m)
+            check_rows(bits, b_ref, M, ldw, W, "bits " + what)
+            assert np.array_equal(u32(vote)[:W], v_ref), what
+            assert np.all(u32(vote)[W:] == np.uint32(0xDEADBEEF)), what
+            gx = f32(xd)
+            assert_same_f32(gx[:d], x_ref, "x " + what)
+            assert np.all(gx[d:] == np.float32(CANARY_F)), what
             if with_m:
-                assert_same_f32(f32(md).reshape(-1), m_ref, "m")
+                assert_same_f32(f32(md).reshape(-1), m_ref, "m " + what)       # includes the untouched elements >= d
 
 
 # Odd vector lengths large enough that the launchers pick their largest tiles (16 and 32 elements per
