@@ -488,7 +488,7 @@ ssgd_status run_step(const StepArgs& a, cudaStream_t s) {
   DeviceInfo di;
   if (!device_info(&di)) return SSGD_ERR_CUDA;
   // short vectors: one launch whose warps work on different rows at once (step_rows.cuh)
-  if (step_uses_rows_kernel(a.M, a.d, di.sms, MODE != kSignSGD)) return launch_step_rows<MODE>(a, s);
+  if (step_uses_rows_kernel(a.M, a.d, di.sms)) return launch_step_rows<MODE>(a, s);
   bool launched = false;
   ssgd_status st = launch_fused<MODE>(a, s, &launched);
   if (st != SSGD_OK || launched) return st;
@@ -608,7 +608,7 @@ ssgd_status ssgd_signsgd_step(float* x, const float* g, float* m, size_t M, size
 int ssgd_step_is_fused(size_t M, size_t d, int momentum) {
   DeviceInfo di;
   if (M < 1 || M > SSGD_MAX_WORKERS || d == 0 || !device_info(&di)) return 0;
-  if (step_uses_rows_kernel(M, d, di.sms, momentum != 0)) return 2;
+  if (step_uses_rows_kernel(M, d, di.sms)) return 2;
   return (momentum ? step_is_fused<kSignum>(M, d, di.sms) : step_is_fused<kSignSGD>(M, d, di.sms)) ? 1 : 0;
 }
 

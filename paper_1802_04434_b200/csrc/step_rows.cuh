@@ -13,6 +13,8 @@
 // Per parameter it moves what fused_step_kernel moves: 12.125 M + 8.125 bytes (4.125 M + 8.125 without a
 // momentum).  Each thread has only two to eight 128-bit loads in flight, so it is the slower kernel as
 // soon as bandwidth matters; the host uses it below a measured number of tiles (see step_rows_max_tiles).
+// The launch bounds hold the register allocation to 48 / 64 / 85 registers for RIF = 1 / 2 / 4 (5 / 4 / 3
+// resident CTAs per SM), which is what its range on the middling sizes depends on.
 #ifndef SSGD_STEP_ROWS_CUH_
 #define SSGD_STEP_ROWS_CUH_
 
@@ -35,7 +37,7 @@ __device__ __forceinline__ void store4_below(float* p, unsigned long long e, uns
 }
 
 template <int MODE, int NP, int RIF>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, RIF <= 1 ? 5 : (RIF == 2 ? 4 : (NP >= 6 ? 2 : 3)))
 step_rows_kernel(const float* __restrict__ g, float* __restrict__ m, float* __restrict__ x,
                  uint32_t* __restrict__ bits, uint32_t* __restrict__ vote, unsigned M,
                  unsigned long long d, unsigned long long ld, unsigned long long ldw, float beta,
@@ -122,22 +124,26 @@ step_rows_kernel(const float* __restrict__ g, float* __restrict__ m, float* __re
 
 // Tiles (of 128 columns) up to which the row-parallel kernel is the faster form of the step, stated per SM
 // of the device.  Measured on B200 (148 SMs; 512 tiles are d = 2^16) against fused_step_kernel (M <= 8)
-// and against worker + vote + apply, every M below at d = 2^10 .. 2^21:
+// and against worker + vote + apply, with and without a momentum (the crossovers agree), d = 2^10 .. 2^21:
 //   one worker: never (the fused kernel is then a single round trip itself);
-//   with a momentum: M = 2 up to d = 2^16, M = 3 .. 6 up to 2^17, M = 7, 8 up to 2^18 (e.g. M = 8 at 2^16:
-//   4.1 us against 11.0), M = 9 .. 32 up to 2^16 (M = 31 at 2^14: 4.8 us against 7.9);
-//   without one: M = 2 up to 2^16, M = 3 .. 16 up to 2^17, M = 17 .. 32 up to 2^16.
-inline unsigned long long step_rows_max_tiles(size_t M, int sms, bool momentum) {
+//   M = 2 up to d = 2^16; M = 3 .. 5 up to 2^17; M = 6 .. 8 up to 2^18; M = 9 .. 16 up to 2^17;
+//   M = 17 .. 32 up to 2^16.
+// Examples, us per step, this kernel against the other form: M = 8, d = 2^16: 4.1 / 10.8; M = 3, d = 2^15:
+// 2.1 / 3.0; M = 16, d = 2^16: 5.3 / 7.8; M = 31, d = 2^14: 4.9 / 7.9.  One size further up it loses: each
+// thread has too few loads in flight to compete once bandwidth matters (M = 7, d = 2^20: 26 / 17).
+inline unsigned long long step_rows_max_tiles(size_t M, int sms) {
   unsigned per_sm;
   if (M <= 1) per_sm = 0;
   else if (M == 2) per_sm = 4;
-  else if (momentum) per_sm = M <= 6 ? 8 : (M <= 8 ? 16 : 4);
-  else per_sm = M <= 16 ? 8 : 4;
+  else if (M <= 5) per_sm = 8;
+  else if (M <= 8) per_sm = 16;
+  else if (M <= 16) per_sm = 8;
+  else per_sm = 4;
   return (unsigned long long)per_sm * (unsigned long long)sms;
 }
 
-inline bool step_uses_rows_kernel(size_t M, size_t d, int sms, bool momentum) {
-  return M <= (size_t)kRowsKernelMaxWorkers && (d + 127) / 128 <= step_rows_max_tiles(M, sms, momentum);
+inline bool step_uses_rows_kernel(size_t M, size_t d, int sms) {
+  return M <= (size_t)kRowsKernelMaxWorkers && (d + 127) / 128 <= step_rows_max_tiles(M, sms);
 }
 
 template <int MODE, int NP, int RIF>
