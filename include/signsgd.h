@@ -109,7 +109,11 @@ ssgd_status ssgd_sign_apply(float* x, const uint32_t* vote, size_t d,
  *   m        in/out [M][ld]; may be NULL only when beta == 0, which selects
  *                   Algorithm 3 as printed (workers send sign(g), no momentum)
  *   bits_ws  out    [M][ldw] workspace: holds the workers' wire words on return
- *   vote_ws  out    [W]      workspace: holds the server's wire words on return */
+ *   vote_ws  out    [W]      workspace: holds the server's wire words on return
+ * Depending on M and d the step is issued as one kernel or as the worker, vote
+ * and apply kernels (ssgd_step_is_fused tells which); in the second form the
+ * vote and apply kernels are launched as programmatic dependents of the kernel
+ * before them, all on `stream`.  The results do not depend on the form.        */
 ssgd_status ssgd_signsgd_step(float* x, const float* g, float* m, size_t M,
                               size_t d, size_t ld, float beta, float delta,
                               uint32_t* bits_ws, size_t ldw, uint32_t* vote_ws,

@@ -572,6 +572,39 @@ def test_resume_from_copied_state_is_bit_identical():
     assert torch.equal(xa, xb) and torch.equal(ma, mb)
 
 
+@pytest.mark.parametrize("M,d", [(12, 600_007), (16, 3_000_017), (9, 20_011), (5, 300_001)])
+def test_step_on_a_side_stream_beside_other_work(M, d):
+    """The step on a stream of its own while the default stream is busy with unrelated kernels: its kernels
+    (vote and apply are programmatic dependents of the kernel before them on THAT stream) must order among
+    themselves alone.  Several steps back to back, then one comparison with the oracle."""
+    ld, W = wl.round_up(d, 4), oracle.words(d)
+    ldw = wl.round_up(W, 4)
+    steps = 3
+    gs = [big_inputs(M, d, ld, seed=100 * k + M)[0] for k in range(steps)]
+    _, m, x = big_inputs(M, d, ld, seed=M + 17)
+    gd = [torch.from_numpy(g).to(DEV) for g in gs]
+    md, xd = torch.from_numpy(m).to(DEV), torch.from_numpy(x[:d].copy()).to(DEV)
+    bits = torch.zeros(M, ldw, dtype=torch.int32, device=DEV)
+    vote = torch.zeros(W, dtype=torch.int32, device=DEV)
+    between, beside = torch.randn(1 << 22, device=DEV), torch.randn(1 << 24, device=DEV)
+    side = torch.cuda.Stream(device=DEV)
+    torch.cuda.synchronize()
+    with torch.cuda.stream(side):
+        for k in range(steps):
+            between.mul_(1.0001)                    # a foreign kernel on the side stream between two steps
+            B.signsgd_step(xd, gd[k], md, M, d, ld, 0.9, 1e-3, bits, ldw, vote, side)
+    for _ in range(20):
+        beside.add_(1.0)                            # the default stream, unordered with the side stream
+    torch.cuda.synchronize()
+    m_ref, x_ref = m.copy().reshape(-1), x[:d].copy()
+    for k in range(steps):
+        b_ref, v_ref = oracle.signsgd_step(x_ref, gs[k].reshape(-1), m_ref, M, d, 0.9, 1e-3, ld=ld, ldw=ldw)
+    assert np.array_equal(u32(bits).reshape(-1), b_ref)
+    assert np.array_equal(u32(vote), v_ref)
+    assert_same_f32(f32(xd), x_ref, "x")
+    assert_same_f32(f32(md).reshape(-1), m_ref, "m")
+
+
 @pytest.mark.parametrize("M,d", [(5, 300_001), (12, 600_007)])
 def test_step_replayed_from_a_cuda_graph(M, d):
     """The step entry point allocates nothing and never synchronises, so a caller can capture it into a CUDA
