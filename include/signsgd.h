@@ -32,7 +32,11 @@
  *     multiples of 4 with ld >= d and ldw >= W (so every row is 16-byte
  *     aligned); 1 <= M <= SSGD_MAX_WORKERS;
  *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream);
- *     work is enqueued on it and the call returns without waiting;
+ *     work is enqueued on it and the call returns without waiting.  Stream
+ *     order holds as for any kernel; the kernels of Algorithms 1-3 are
+ *     launched as programmatic dependents of the kernel before them on the
+ *     stream, i.e. they may be brought onto the GPU while that kernel drains,
+ *     but touch no memory before it has completed;
  *   - d == 0 is valid: nothing is launched, SSGD_OK is returned;
  *   - buffers must not overlap except where "in place" is stated;
  *   - arguments are checked on the host before anything is launched; a failed
@@ -111,9 +115,8 @@ ssgd_status ssgd_sign_apply(float* x, const uint32_t* vote, size_t d,
  *   bits_ws  out    [M][ldw] workspace: holds the workers' wire words on return
  *   vote_ws  out    [W]      workspace: holds the server's wire words on return
  * Depending on M and d the step is issued as one kernel or as the worker, vote
- * and apply kernels (ssgd_step_is_fused tells which); in the second form the
- * vote and apply kernels are launched as programmatic dependents of the kernel
- * before them, all on `stream`.  The results do not depend on the form.        */
+ * and apply kernels, all on `stream` (ssgd_step_is_fused tells which).  The
+ * results do not depend on the form.                                           */
 ssgd_status ssgd_signsgd_step(float* x, const float* g, float* m, size_t M,
                               size_t d, size_t ld, float beta, float delta,
                               uint32_t* bits_ws, size_t ldw, uint32_t* vote_ws,

@@ -63,8 +63,8 @@ inline bool beta_ok(float beta) { return beta >= 0.0f && beta < 1.0f; }  // fals
 
 ssgd_status launch_status() { return cudaGetLastError() == cudaSuccess ? SSGD_OK : SSGD_ERR_CUDA; }
 
-// Kernel launch with or without the programmatic-serialization attribute (see pdl_wait in
-// device_common.cuh).  Only kernels that begin with pdl_wait() may be launched with it.
+// Kernel launch with the programmatic-serialization attribute (see pdl_wait in device_common.cuh), for
+// kernels that begin with pdl_wait(); pdl = false gives an ordinary launch.
 template <typename... KArgs, typename... Args>
 void launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, bool pdl,
                    Args... args) {

@@ -77,7 +77,8 @@ worker_pack_kernel(const float* __restrict__ g, float* __restrict__ m,
   constexpr bool SIGN_OF_G = MODE != kSignum;
   constexpr unsigned long long TILE = (unsigned long long)kThreads * 4 * UNROLL;
   constexpr unsigned SPAN = 128 * UNROLL;
-  pdl_launch_dependents();   // in a step the vote kernel may be brought in while this grid drains
+  pdl_launch_dependents();
+  pdl_wait();
   const unsigned lane = threadIdx.x & 31u;
   const unsigned warp = threadIdx.x >> 5;
   const unsigned long long row = blockIdx.y;
@@ -159,7 +160,8 @@ __device__ __forceinline__ void apply_ragged_span(float* __restrict__ x, const u
 template <int UNROLL, bool RAGGED>
 __global__ void __launch_bounds__(kThreads, 1)
 apply_kernel(float* __restrict__ x, const uint32_t* __restrict__ vote, unsigned long long d, float delta) {
-  pdl_wait();   // the vote may come from the kernel before this one on the stream
+  pdl_launch_dependents();
+  pdl_wait();
   constexpr unsigned long long TILE = (unsigned long long)kThreads * 4 * UNROLL;
   constexpr unsigned SPAN = 128 * UNROLL;
   const unsigned lane = threadIdx.x & 31u;
@@ -316,6 +318,8 @@ fused_step_kernel(const float* __restrict__ g, float* __restrict__ m, float* __r
   const unsigned lane = threadIdx.x & 31u;
   const unsigned warp = threadIdx.x >> 5;
   const unsigned sub = lane & 7u;
+  pdl_launch_dependents();
+  pdl_wait();
   const unsigned long long e0 = (unsigned long long)blockIdx.x * TILE + (unsigned long long)warp * SPAN;
   if (e0 >= d) return;   // uniform over the warp; nothing below synchronises across warps
   if (e0 + SPAN > d) {
@@ -349,8 +353,8 @@ fused_step_kernel(const float* __restrict__ g, float* __restrict__ m, float* __r
 // host side
 
 ssgd_status launch_vote(const uint32_t* bits, size_t M, size_t d, size_t ldw, uint32_t* vote,
-                        cudaStream_t s, bool pdl = false) {
-  return launch_vote_any<false>(bits, M, d, ldw, vote, 0, s, pdl);
+                        cudaStream_t s) {
+  return launch_vote_any<false>(bits, M, d, ldw, vote, 0, s);
 }
 
 constexpr size_t kWorkerSharedHint = 36 * 1024;   // below the 48 KB that need no opt-in
@@ -368,8 +372,8 @@ bool launch_worker_u(const float* g, float* m, size_t M, size_t d, size_t ld, fl
   // measured on B200 (d = 335 M, M = 16, five runs on different boards) the stream is then 0.7-1.3 %
   // faster than with the whole array as L1, while 170 KB and more on the shared side is slower.
   const size_t smem = SPLIT ? kWorkerSharedHint : 0;
-  worker_pack_kernel<MODE, UNROLL, !SPLIT><<<dim3((unsigned)tiles_per_row, (unsigned)M), kThreads, smem, s>>>(
-      g, m, bits, d, ld, ldw, beta, omb);
+  launch_kernel(worker_pack_kernel<MODE, UNROLL, !SPLIT>, dim3((unsigned)tiles_per_row, (unsigned)M), kThreads, smem, s,
+                true, g, m, bits, (unsigned long long)d, (unsigned long long)ld, (unsigned long long)ldw, beta, omb);
   if constexpr (SPLIT) {
     if (d % (128 * UNROLL) != 0)
       worker_tail_kernel<MODE, UNROLL><<<(unsigned)M, 32, 0, s>>>(g, m, bits, d, ld, ldw, beta, omb);
@@ -398,11 +402,11 @@ ssgd_status launch_worker(const float* g, float* m, size_t M, size_t d, size_t l
 }
 
 template <int UNROLL, bool SPLIT>
-bool launch_apply_u(float* x, const uint32_t* vote, size_t d, float delta, cudaStream_t s, bool pdl) {
+bool launch_apply_u(float* x, const uint32_t* vote, size_t d, float delta, cudaStream_t s) {
   constexpr unsigned long long TILE = (unsigned long long)kThreads * 4 * UNROLL;
   const unsigned long long tiles = (d + TILE - 1) / TILE;
   if (tiles > kMaxGrid) return false;     // beyond any device's memory
-  launch_kernel(apply_kernel<UNROLL, !SPLIT>, (unsigned)tiles, kThreads, 0, s, pdl, x, vote,
+  launch_kernel(apply_kernel<UNROLL, !SPLIT>, (unsigned)tiles, kThreads, 0, s, true, x, vote,
                 (unsigned long long)d, delta);
   if constexpr (SPLIT) {
     if (d % (128 * UNROLL) != 0) apply_tail_kernel<UNROLL><<<1, 32, 0, s>>>(x, vote, d, delta);
@@ -410,14 +414,13 @@ bool launch_apply_u(float* x, const uint32_t* vote, size_t d, float delta, cudaS
   return true;
 }
 
-ssgd_status launch_apply(float* x, const uint32_t* vote, size_t d, float delta, cudaStream_t s,
-                         bool pdl = false) {
+ssgd_status launch_apply(float* x, const uint32_t* vote, size_t d, float delta, cudaStream_t s) {
   DeviceInfo di;
   if (!device_info(&di)) return SSGD_ERR_CUDA;
   // 2048-element tiles, interior-only, once they fill the machine 8 CTAs deep; below that the smallest
   // tile with the guarded path inline (one launch)
-  const bool ok = apply_unroll(d, di.sms) == 2 ? launch_apply_u<2, true>(x, vote, d, delta, s, pdl)
-                                               : launch_apply_u<1, false>(x, vote, d, delta, s, pdl);
+  const bool ok = apply_unroll(d, di.sms) == 2 ? launch_apply_u<2, true>(x, vote, d, delta, s)
+                                               : launch_apply_u<1, false>(x, vote, d, delta, s);
   return ok ? launch_status() : SSGD_ERR_SIZE;
 }
 
@@ -425,9 +428,9 @@ template <int MODE, int UNROLL, int NP>
 void launch_fused_mun(const StepArgs& a, cudaStream_t s) {
   constexpr unsigned long long TILE = (unsigned long long)kThreads * 4 * UNROLL;
   const unsigned long long tiles = (a.d + TILE - 1) / TILE;
-  fused_step_kernel<MODE, UNROLL, NP><<<(unsigned)tiles, kThreads, 0, s>>>(
-      a.g, a.m, a.x, a.bits, a.vote, (unsigned)a.M, a.d, a.ld, a.ldw, a.beta, 1.0f - a.beta, a.delta,
-      vote_start_value(a.M, NP));
+  launch_kernel(fused_step_kernel<MODE, UNROLL, NP>, (unsigned)tiles, kThreads, 0, s, true, a.g, a.m, a.x, a.bits,
+                a.vote, (unsigned)a.M, (unsigned long long)a.d, (unsigned long long)a.ld, (unsigned long long)a.ldw,
+                a.beta, 1.0f - a.beta, a.delta, vote_start_value(a.M, NP));
 }
 
 template <int MODE, int UNROLL>
@@ -494,11 +497,11 @@ ssgd_status run_step(const StepArgs& a, cudaStream_t s) {
   if (st != SSGD_OK || launched) return st;
   st = launch_worker<MODE>(a.g, a.m, a.M, a.d, a.ld, a.beta, a.bits, a.ldw, s);
   if (st != SSGD_OK) return st;
-  // vote and apply follow this library's own kernels on the stream: programmatic dependent launch lets
-  // each be brought onto the SMs while its predecessor drains (both begin with pdl_wait())
-  st = launch_vote(a.bits, a.M, a.d, a.ldw, a.vote, s, true);
+  // programmatic dependent launches: vote and apply are each brought onto the SMs while the kernel before
+  // them drains (see pdl_wait)
+  st = launch_vote(a.bits, a.M, a.d, a.ldw, a.vote, s);
   if (st != SSGD_OK) return st;
-  return launch_apply(a.x, a.vote, a.d, a.delta, s, true);
+  return launch_apply(a.x, a.vote, a.d, a.delta, s);
 }
 
 // argument checks shared by the entry points -------------------------------

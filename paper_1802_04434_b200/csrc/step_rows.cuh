@@ -46,6 +46,8 @@ step_rows_kernel(const float* __restrict__ g, float* __restrict__ m, float* __re
   constexpr bool SIGN_OF_G = MODE != kSignum;
   constexpr unsigned kWarps = kThreads / 32;
   __shared__ unsigned part[kWarps][NP][4];   // partial counts: [warp][plane][word of the tile]
+  pdl_launch_dependents();
+  pdl_wait();
   const unsigned lane = threadIdx.x & 31u;
   const unsigned warp = threadIdx.x >> 5;
   const unsigned group = lane >> 3;          // which of the tile's four words this lane's bits go to
@@ -149,9 +151,9 @@ inline bool step_uses_rows_kernel(size_t M, size_t d, int sms) {
 template <int MODE, int NP, int RIF>
 void launch_step_rows_np(const StepArgs& a, cudaStream_t s) {
   const unsigned tiles = (unsigned)((a.d + 127) / 128);
-  step_rows_kernel<MODE, NP, RIF><<<tiles, kThreads, 0, s>>>(a.g, a.m, a.x, a.bits, a.vote, (unsigned)a.M, a.d, a.ld,
-                                                          a.ldw, a.beta, 1.0f - a.beta, a.delta,
-                                                          vote_start_value(a.M, NP));
+  launch_kernel(step_rows_kernel<MODE, NP, RIF>, tiles, kThreads, 0, s, true, a.g, a.m, a.x, a.bits, a.vote,
+                (unsigned)a.M, (unsigned long long)a.d, (unsigned long long)a.ld, (unsigned long long)a.ldw, a.beta,
+                1.0f - a.beta, a.delta, vote_start_value(a.M, NP));
 }
 
 template <int MODE>

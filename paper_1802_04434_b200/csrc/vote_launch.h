@@ -30,11 +30,10 @@ unsigned count_planes(size_t M) {
   return n;
 }
 
-// pdl: launch with the programmatic-serialization attribute (the step entry points, where the kernel
-// before this one on the stream is this library's own).
 template <bool COUNTS>
 ssgd_status launch_vote_any(const uint32_t* bits, size_t M, size_t d, size_t ldw, uint32_t* out,
-                            size_t ldc, cudaStream_t s, bool pdl = false) {
+                            size_t ldc, cudaStream_t s) {
+  const bool pdl = true;   // vote_kernel begins with pdl_wait()
   DeviceInfo di;
   if (!device_info(&di)) return SSGD_ERR_CUDA;
   const size_t W = ssgd_words(d);
