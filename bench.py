@@ -43,15 +43,15 @@ FALLBACK_HBM_GBS = 6650.0
 # with the same M it is scaled (the path is elementwise, so traffic grows in proportion to d as long as
 # the operands exceed L2).  Valid only while the kernel sources are unchanged.
 NCU_TRAFFIC = {
-    "source_sha256": "8581929ce5634a8b9845b6cdc91d07387422d2f94e26ed1ced4f45bc563ad5be",
+    "source_sha256": "8954f1d9109e82c54c7fced02c37cbd4ea71feadea3a30168d2bd186298b74c0",
     "per_param": {
         # profiles/dram_bytes_worker_vote_apply_bertlarge_M16_full_size.md: a one-pass capture of the full-size
         # default workload (d = 335,141,888)
-        "worker_pack_kernel:M16": {"bytes_per_param": (42898985216 + 22068073728) / 335141888, "d": 335141888},
-        "vote_kernel:M16": {"bytes_per_param": (670295296 + 36635904) / 335141888, "d": 335141888},
-        "apply_kernel:M16": {"bytes_per_param": (1382499328 + 1277744640) / 335141888, "d": 335141888},
+        "worker_pack_kernel:M16": {"bytes_per_param": (42900414720 + 22067966720) / 335141888, "d": 335141888},
+        "vote_kernel:M16": {"bytes_per_param": (670294528 + 36479744) / 335141888, "d": 335141888},
+        "apply_kernel:M16": {"bytes_per_param": (1382476032 + 1277456128) / 335141888, "d": 335141888},
         # profiles/fused_step_kernel_resnet50_M7_ncu_full.md (captured at full size)
-        "fused_step_kernel:M7": {"bytes_per_param": (1.533654e9 + 794.602496e6) / 25557056, "d": 25557056},
+        "fused_step_kernel:M7": {"bytes_per_param": (1.533654e9 + 793.715968e6) / 25557056, "d": 25557056},
     },
 }
 
