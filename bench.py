@@ -43,15 +43,15 @@ FALLBACK_HBM_GBS = 6650.0
 # with the same M it is scaled (the path is elementwise, so traffic grows in proportion to d as long as
 # the operands exceed L2).  Valid only while the kernel sources are unchanged.
 NCU_TRAFFIC = {
-    "source_sha256": "8954f1d9109e82c54c7fced02c37cbd4ea71feadea3a30168d2bd186298b74c0",
+    "source_sha256": "0a866e07409fea43f5c7caec69a60af5f41d350a244bbfbe6da7f1ffba79e190",
     "per_param": {
         # profiles/dram_bytes_worker_vote_apply_bertlarge_M16_full_size.md: a one-pass capture of the full-size
         # default workload (d = 335,141,888)
-        "worker_pack_kernel:M16": {"bytes_per_param": (42900414720 + 22067966720) / 335141888, "d": 335141888},
-        "vote_kernel:M16": {"bytes_per_param": (670294528 + 36479744) / 335141888, "d": 335141888},
-        "apply_kernel:M16": {"bytes_per_param": (1382476032 + 1277456128) / 335141888, "d": 335141888},
+        "worker_pack_kernel:M16": {"bytes_per_param": (42898779904 + 22067552000) / 335141888, "d": 335141888},
+        "vote_kernel:M16": {"bytes_per_param": (670358016 + 36536064) / 335141888, "d": 335141888},
+        "apply_kernel:M16": {"bytes_per_param": (1382519296 + 1278086144) / 335141888, "d": 335141888},
         # profiles/fused_step_kernel_resnet50_M7_ncu_full.md (captured at full size)
-        "fused_step_kernel:M7": {"bytes_per_param": (1.533654e9 + 793.715968e6) / 25557056, "d": 25557056},
+        "fused_step_kernel:M7": {"bytes_per_param": (1.533640e9 + 793.140480e6) / 25557056, "d": 25557056},
     },
 }
 
@@ -460,6 +460,10 @@ def host_buffer(torch, shape, dtype):
         return torch.empty(shape, dtype=dtype), "pageable"
 
 
+class _SkipE2E(Exception):
+    """--e2e-steps 0."""
+
+
 def run_ours(args):
     import torch
     from paper_1802_04434_b200 import binding as B
@@ -521,6 +525,8 @@ def run_ours(args):
     Ke = max(1, min(K, args.e2e_steps))
     e2e = None
     try:
+        if args.e2e_steps <= 0:                      # profiling runs that want the step's kernels only
+            raise _SkipE2E
         g_host, host_kind = host_buffer(torch, (M, ld), torch.float32)
         g_host.copy_(b.g)
         vote_host, _ = host_buffer(torch, (W,), torch.int32)
@@ -541,6 +547,10 @@ def run_ours(args):
                "entry_point": "ssgd_signsgd_step_host",
                "h2d_gbs": M * ld * 4 / (e2e_ms / Ke * 1e-3) / 1e9}
         del g_host, vote_host
+    except _SkipE2E:
+        e2e = {"value": None, "unit": UNIT, "h2d_bytes_per_step": M * ld * 4, "d2h_bytes_per_step": W * 4,
+               "skipped": "--e2e-steps 0"}
+        multi.barrier(dev)
     except (RuntimeError, MemoryError) as exc:   # the host could not hold one step's gradients
         e2e = {"value": None, "unit": UNIT, "h2d_bytes_per_step": M * ld * 4, "d2h_bytes_per_step": W * 4,
                "error": "host buffer of %.1f GB not granted: %s" % (M * ld * 4 / 1e9, str(exc)[:120])}
@@ -709,8 +719,8 @@ def main():
     ap.add_argument("--exchange", choices=["allgather", "p2p"], default="allgather",
                     help="--mode workers: how the sign rows travel (a collective, or peer stores from the worker kernel)")
     ap.add_argument("--seed", type=int, default=0)
-    ap.add_argument("--e2e-steps", type=int, default=3)
-    ap.add_argument("--e2e-warmup", type=int, default=1)
+    ap.add_argument("--e2e-steps", type=int, default=3, help="timed end-to-end steps (0: skip the end-to-end leg)")
+    ap.add_argument("--e2e-warmup", type=int, default=3)
     ap.add_argument("--ref-threads", type=int, default=0, help="threads of the oracle arm (0 = all host cores)")
     ap.add_argument("--ref-sample", type=int, default=0,
                     help="parameters per step of the oracle arm (0 = sized from a probe of its speed)")

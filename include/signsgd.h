@@ -232,9 +232,18 @@ ssgd_status ssgd_welford_update(const float* g, size_t n, float* mean, float* m2
 /* ssgd_signsgd_step for a caller whose gradients live in HOST memory
  * (Algorithm 3's "independent gradient estimate" arriving from outside the
  * device): copies g_host to the device staging buffer, runs the step, and
- * copies the voted words back to the host, all enqueued on `stream`.
- *   g_host    in   HOST  [M][ld]; page-locked memory makes the copy asynchronous
- *   g_stage   out  DEVICE [M][ld] staging buffer for the gradients
+ * copies the voted words back to the host; everything is ordered after what
+ * `stream` already holds, and complete once `stream` has been synchronised.
+ * A large transfer (128 MB and more of gradients) is cut into up to 32 slabs of
+ * columns, copied by a stream that the call creates and releases, while `stream`
+ * runs the step on the slabs that have arrived (the step is elementwise in the
+ * parameter index, so the results are those of one step on the whole vector);
+ * smaller ones, and calls made while `stream` is being captured, are one copy
+ * and one step on `stream`.
+ *   g_host    in   HOST  [M][ld]; page-locked memory makes the copies
+ *                  asynchronous and lets them overlap the kernels
+ *   g_stage   out  DEVICE [M][ld] staging buffer for the gradients (elements
+ *                  d..ld-1 of its rows may be left unwritten)
  *   vote_host out  HOST  [W] (may be NULL: no copy back); valid once `stream`
  *                  has been synchronised
  *   x, m, bits_ws, vote_ws: DEVICE, as in ssgd_signsgd_step.                   */

@@ -686,14 +686,62 @@ ssgd_status ssgd_signsgd_step_host(float* x, const float* g_host, float* m, size
   ssgd_status st = check_step(x, g_stage, m, M, d, ld, beta, delta, bits_ws, ldw, vote_ws);
   if (st != SSGD_OK || d == 0) return st;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  if (cudaMemcpyAsync(g_stage, g_host, M * ld * sizeof(float), cudaMemcpyHostToDevice, s) != cudaSuccess)
-    return SSGD_ERR_CUDA;
-  st = ssgd_signsgd_step(x, g_stage, m, M, d, ld, beta, delta, bits_ws, ldw, vote_ws, stream);
+  const size_t vote_bytes = ssgd_words(d) * sizeof(uint32_t);
+
+  // The step is elementwise in the parameter index, so a slab of columns can be stepped as soon as it
+  // has arrived.  Large transfers are therefore cut into column slabs that a second stream copies while
+  // `stream` computes on the slabs before them; the host link stays busy throughout and only the last
+  // slab's kernels are left over at the end.  Slab starts are multiples of 4096 parameters (whole words,
+  // 16-byte aligned rows).  Small transfers, and calls under stream capture, take one copy and one step.
+  constexpr size_t kSlabBytes = size_t(64) << 20;
+  constexpr size_t kMaxSlabs = 32;
+  const size_t total = M * d * sizeof(float);
+  size_t slabs = total / kSlabBytes;
+  if (slabs > kMaxSlabs) slabs = kMaxSlabs;
+  cudaStreamCaptureStatus capturing = cudaStreamCaptureStatusNone;
+  if (cudaStreamIsCapturing(s, &capturing) != cudaSuccess) return SSGD_ERR_CUDA;
+  if (slabs < 2 || capturing != cudaStreamCaptureStatusNone) {
+    if (cudaMemcpyAsync(g_stage, g_host, M * ld * sizeof(float), cudaMemcpyHostToDevice, s) != cudaSuccess)
+      return SSGD_ERR_CUDA;
+    st = ssgd_signsgd_step(x, g_stage, m, M, d, ld, beta, delta, bits_ws, ldw, vote_ws, stream);
+    if (st != SSGD_OK) return st;
+    if (vote_host && cudaMemcpyAsync(vote_host, vote_ws, vote_bytes, cudaMemcpyDeviceToHost, s) != cudaSuccess)
+      return SSGD_ERR_CUDA;
+    return SSGD_OK;
+  }
+
+  const size_t width = ((d + slabs - 1) / slabs + 4095) / 4096 * 4096;   // parameters per slab
+  cudaStream_t copier = nullptr;
+  cudaEvent_t ready[kMaxSlabs + 1] = {};                                  // [slabs]: `stream`'s earlier work
+  size_t events = 0;
+  bool ok = cudaStreamCreateWithFlags(&copier, cudaStreamNonBlocking) == cudaSuccess;
+  for (; ok && events <= slabs; ++events)
+    ok = cudaEventCreateWithFlags(&ready[events], cudaEventDisableTiming) == cudaSuccess;
+  // the copies may not overwrite g_stage before what `stream` already holds has run
+  ok = ok && cudaEventRecord(ready[slabs], s) == cudaSuccess &&
+       cudaStreamWaitEvent(copier, ready[slabs], 0) == cudaSuccess;
+  st = SSGD_OK;
+  size_t k = 0;
+  for (size_t off = 0; ok && st == SSGD_OK && off < d; off += width, ++k) {
+    const size_t w = d - off < width ? d - off : width;
+    ok = cudaMemcpy2DAsync(g_stage + off, ld * sizeof(float), g_host + off, ld * sizeof(float), w * sizeof(float), M,
+                           cudaMemcpyHostToDevice, copier) == cudaSuccess &&
+         cudaEventRecord(ready[k], copier) == cudaSuccess && cudaStreamWaitEvent(s, ready[k], 0) == cudaSuccess;
+    if (ok)
+      st = ssgd_signsgd_step(x + off, g_stage + off, m ? m + off : nullptr, M, w, ld, beta, delta, bits_ws + off / 32,
+                             ldw, vote_ws + off / 32, stream);
+  }
+  if (ok && st == SSGD_OK && vote_host)
+    ok = cudaMemcpyAsync(vote_host, vote_ws, vote_bytes, cudaMemcpyDeviceToHost, s) == cudaSuccess;
+  // events and the stream may be destroyed while their work is still queued: the runtime releases them
+  // once it has completed
+  for (size_t e = 0; e < events; ++e) (void)cudaEventDestroy(ready[e]);
+  if (copier) (void)cudaStreamDestroy(copier);
   if (st != SSGD_OK) return st;
-  if (vote_host &&
-      cudaMemcpyAsync(vote_host, vote_ws, ssgd_words(d) * sizeof(uint32_t), cudaMemcpyDeviceToHost, s) !=
-          cudaSuccess)
+  if (!ok) {
+    (void)cudaGetLastError();
     return SSGD_ERR_CUDA;
+  }
   return SSGD_OK;
 }
 

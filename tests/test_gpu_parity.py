@@ -553,6 +553,43 @@ def test_host_buffer_step_matches_device_step():
     assert torch.equal(vote1.cpu(), vote_host)
 
 
+@pytest.mark.parametrize("M,d,beta", [(5, 8_000_003, 0.9), (12, 6_000_007, 0.9), (3, 24_000_001, 0.0)])
+def test_host_buffer_step_in_column_slabs(M, d, beta):
+    """Transfers of 128 MB and more are cut into column slabs that a second stream copies while the step runs on
+    the slabs before them.  Two calls in a row with different gradients through the SAME staging buffer (the second
+    call's copies must wait for the first call's kernels), against two device steps; x starts from a canary tail."""
+    ld, W = wl.round_up(d, 4) + 4, oracle.words(d)
+    ldw = wl.round_up(W, 4) + 4
+    gen = torch.Generator().manual_seed(M * 1000 + d % 997)
+    g_host = [torch.randn(M, ld, generator=gen).pin_memory() for _ in range(2)]
+    x0 = torch.randn(d + 8, generator=gen)
+    x0[d:] = CANARY_F
+    with_m = beta != 0.0
+    xs, ms, bs, vs = [], [], [], []
+    for _ in range(2):
+        xs.append(x0.to(DEV))
+        ms.append(torch.zeros(M, ld, device=DEV) if with_m else None)
+        bs.append(torch.full((M, ldw), CANARY_WORD, dtype=torch.int32, device=DEV))
+        vs.append(torch.full((W + 4,), CANARY_WORD, dtype=torch.int32, device=DEV))
+    stage = torch.full((M, ld), float("nan"), device=DEV)
+    vote_host = [torch.zeros(W, dtype=torch.int32).pin_memory() for _ in range(2)]
+    votes_dev = []
+    for k in range(2):
+        B.signsgd_step(xs[0], g_host[k].to(DEV), ms[0], M, d, ld, beta, 1e-3, bs[0], ldw, vs[0])
+        votes_dev.append(vs[0][:W].clone())
+    for k in range(2):                                   # back to back, no synchronisation in between
+        B.signsgd_step_host(xs[1], g_host[k], ms[1], M, d, ld, beta, 1e-3, stage, bs[1], ldw, vs[1], vote_host[k])
+    torch.cuda.synchronize()
+    assert torch.equal(xs[0].view(torch.int32), xs[1].view(torch.int32))
+    assert torch.equal(bs[0], bs[1]) and torch.equal(vs[0], vs[1])
+    if with_m:
+        assert torch.equal(ms[0].view(torch.int32), ms[1].view(torch.int32))
+    for k in range(2):
+        assert torch.equal(votes_dev[k].cpu(), vote_host[k]), "voted words of call %d" % k
+    assert np.all(u32(vs[1])[W:] == np.uint32(0xDEADBEEF)) and np.all(f32(xs[1])[d:] == np.float32(CANARY_F))
+    assert np.all(u32(bs[1])[:, W:] == np.uint32(0xDEADBEEF))
+
+
 def test_resume_from_copied_state_is_bit_identical():
     cfg = wl.small_signum(d=50_000, M=3)
     M, d, ld, ldw, W = cfg.M, cfg.d, cfg.ld, cfg.ldw, cfg.words
