@@ -14,7 +14,8 @@
 // momentum).  Each thread has only two to eight 128-bit loads in flight, so it is the slower kernel as
 // soon as bandwidth matters; the host uses it below a measured number of tiles (see step_rows_max_tiles).
 // The launch bounds hold the register allocation to 48 / 64 / 85 registers for RIF = 1 / 2 / 4 (5 / 4 / 3
-// resident CTAs per SM), which is what its range on the middling sizes depends on.
+// resident CTAs per SM; 128 registers for the six-plane form, M = 32, which would spill at 85), which is
+// what its range on the middling sizes depends on.
 #ifndef SSGD_STEP_ROWS_CUH_
 #define SSGD_STEP_ROWS_CUH_
 
