@@ -252,14 +252,14 @@ __device__ __forceinline__ void store_plane_words(uint32_t* __restrict__ out, un
 //                   scheme of Section 4.
 //   GUARDED = false: after the batches of eight rows, the remaining rows come in
 //                   batches of 4, 2 and 1, each loaded and folded in turn (fewest
-//                   registers: 27-32 for M <= 7, so all warp slots fill).
+//                   registers).
 //   GUARDED = true: the remaining rows come as ONE batch of four or eight loads with
 //                   the missing rows as words of zeros, so that a thread makes
 //                   ceil(M / 8) round trips to memory instead of up to three more.
 //                   Measured on B200: a round trip costs a short launch about 0.5 us,
-//                   and this form is 5-20 % faster for M = 15 and 31 at every size and
-//                   for M = 7 up to d = 2^24, but 3-20 % slower for M <= 7 on long
-//                   vectors (42-56 registers); the host picks per launch.
+//                   and this form is 5-20 % faster for M = 15 and 31 at every size;
+//                   the host picks per launch (vote_guarded).
+// Two to seven rows (two and three planes) go to vote_exact_kernel below instead.
 template <int NP, bool COUNTS, bool GUARDED>
 __global__ void __launch_bounds__(kThreads)
 vote_kernel(const uint32_t* __restrict__ bits, unsigned M, unsigned long long d,
@@ -331,6 +331,46 @@ vote_kernel(const uint32_t* __restrict__ bits, unsigned M, unsigned long long d,
         w += 1;
       }
     }
+    if (COUNTS) {
+#pragma unroll
+      for (int p = 0; p < NP; ++p) store_plane_words(out + (unsigned long long)p * ldc, q, d, cnt.c[p]);
+    } else {
+      store_plane_words(out, q, d, cnt.c[NP - 1]);
+    }
+  }
+}
+
+
+// The same vote for exactly MROWS = 2 .. 7 rows (two and three planes): all rows are loaded before the
+// first use, without guards, and folded in one carry-save step, so that a thread makes ONE round trip to
+// memory at 30-36 registers (vote_kernel needs up to three trips for these row counts, or 48-56 registers
+// in its guarded form).  Measured on B200 against vote_kernel: M = 5: 2.66 -> 2.09 us at d = 2^22,
+// 9.00 -> 8.64 at 2^26; M = 7: 20.9 -> 20.2 at 2^27; M = 2, 3: 1-5 % at every size.
+template <int NP, bool COUNTS, int MROWS>
+__global__ void __launch_bounds__(kThreads)
+vote_exact_kernel(const uint32_t* __restrict__ bits, unsigned long long d, unsigned long long W,
+                  unsigned long long ldw, uint32_t* __restrict__ out, unsigned long long ldc,
+                  unsigned start_value) {
+  static_assert(MROWS >= 2 && MROWS <= 7 && NP >= 2 && NP <= 3, "row counts with two or three planes");
+  pdl_launch_dependents();
+  pdl_wait();
+  const unsigned long long chunks = (W + 3) / 4;
+  const unsigned long long stride = (unsigned long long)gridDim.x * kThreads;
+  for (unsigned long long q = (unsigned long long)blockIdx.x * kThreads + threadIdx.x; q < chunks; q += stride) {
+    const uint32_t* col = bits + 4 * q;
+    W4 a[8];
+#pragma unroll
+    for (int k = 0; k < MROWS; ++k) a[k] = ld_words(col + (unsigned long long)k * ldw);
+#pragma unroll
+    for (int k = MROWS; k < 8; ++k) a[k] = W4{0u, 0u, 0u, 0u};   // folded away at compile time
+    Counter<NP> cnt;
+#pragma unroll
+    for (int p = 0; p < NP; ++p) {
+      const unsigned f = ((start_value >> p) & 1u) ? 0xFFFFFFFFu : 0u;
+      cnt.c[p] = W4{f, f, f, f};
+    }
+    if (MROWS <= 4) cnt.fold4(a);
+    else cnt.fold8(a);
     if (COUNTS) {
 #pragma unroll
       for (int p = 0; p < NP; ++p) store_plane_words(out + (unsigned long long)p * ldc, q, d, cnt.c[p]);

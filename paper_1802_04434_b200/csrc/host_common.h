@@ -115,16 +115,13 @@ inline int fused_unroll(unsigned long long d, int sms, bool momentum) {
 inline int apply_unroll(unsigned long long d, int sms) { return tile_count(d, 1, 2) >= 8ull * sms ? 2 : 1; }
 
 // Vote kernel: the remaining rows after the batches of eight come as one guarded batch (see vote_kernel)
-// with four to six planes (M = 8 .. 127: 5-20 % faster at every size measured), and with three planes
-// (M = 4 .. 7) while the launch is at most four CTAs per SM deep (beyond that its 56 registers cost
-// more than the round trips save).  With more planes the kernel makes eight and more round trips
-// anyway and the guarded form would go from 64 to 72-80 registers; with fewer it has nothing to save.
-// Crossovers measured on B200.
-constexpr int kGuardedMinPlanes = 3;
+// with four to six planes (M = 8 .. 127: 5-20 % faster at every size measured).  With more planes the
+// kernel makes eight and more round trips anyway and the guarded form would go from 64 to 72-80
+// registers.  One plane is one row; two and three planes (M = 2 .. 7) have a kernel of their own.
+constexpr int kGuardedMinPlanes = 4;
 constexpr int kGuardedMaxPlanes = 6;
-inline bool vote_guarded(unsigned planes, unsigned long long ctas, int sms) {
-  if (planes == 3) return ctas <= 4ull * sms;
-  return planes > 3 && planes <= (unsigned)kGuardedMaxPlanes;
+inline bool vote_guarded(unsigned planes) {
+  return planes >= (unsigned)kGuardedMinPlanes && planes <= (unsigned)kGuardedMaxPlanes;
 }
 
 unsigned vote_planes(size_t M) {

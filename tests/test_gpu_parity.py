@@ -117,8 +117,9 @@ def test_majority_vote_small(M):
                                  (13, (1 << 24) + 4099), (31, 5_000_003), (63, 2_000_003), (64, 2_000_003),
                                  (100, 1_000_003)])
 def test_majority_vote_long_vectors(M, d):
-    """Both forms of the vote kernel's tail (remaining rows in batches of 4, 2, 1, or as one guarded batch) on
-    launches many CTAs per SM deep and on shorter ones, with a ragged last word and garbage in the row padding."""
+    """The vote kernels (the one for exactly 2 .. 7 rows; the general one with its remaining rows as one guarded
+    batch, M = 8 .. 127, or in batches of 4, 2, 1) on launches many CTAs per SM deep and on shorter ones, with a
+    ragged last word and garbage in the row padding."""
     r = np.random.default_rng(M * 7919 + d % 1000)
     W = oracle.words(d)
     ldw = wl.round_up(W, 4) + 8
