@@ -248,6 +248,49 @@ def test_whole_step_small(M):
                 assert_same_f32(f32(md).reshape(-1), m_ref, "m " + what)       # includes the untouched elements >= d
 
 
+@pytest.mark.parametrize("seed", range(48))
+def test_whole_step_random_shapes(seed):
+    """Seeded random problems across the launch forms of the step (row-parallel, fused with either tile, worker +
+    vote + apply): random worker count, length, row strides and mode (Signum, sign-only, warm-up), two steps each,
+    everything compared with the oracle, canaries behind every output."""
+    r = np.random.default_rng(1000 + seed)
+    M = int(r.choice([1, 2, 3, 4, 5, 6, 7, 8, 9, 12, 15, 16, 17, 24, 31, 32, 33, 40]))
+    d = int(10 ** r.uniform(0.0, 5.6)) if seed % 4 else int(r.choice([65_535, 65_537, 131_073, 262_145, 151_553, 303_105]))
+    mode = ("signum", "sign_only", "warmup")[seed % 3]
+    ld = wl.round_up(d, 4) + 4 * int(r.integers(0, 3))
+    W = oracle.words(d)
+    ldw = wl.round_up(W, 4) + 4 * int(r.integers(0, 3))
+    beta = 0.0 if mode == "sign_only" else float(r.choice([0.5, 0.9, 0.99]))
+    delta = float(r.choice([1e-4, 1e-2, 0.5]))
+    g0, m, x = rand_inputs(M, d, ld, seed=seed, special=True)
+    x = np.concatenate([x[:d], np.full(8, CANARY_F, dtype=np.float32)])
+    with_m = mode != "sign_only"
+    md = torch.from_numpy(m).to(DEV) if with_m else None
+    xd = torch.from_numpy(x).to(DEV)
+    m_ref = m.copy().reshape(-1) if with_m else None
+    x_ref = x[:d].copy()
+    for k in range(2):
+        g = g0 if k == 0 else rand_inputs(M, d, ld, seed=seed + 500)[0]
+        bits = torch.full((M, ldw), CANARY_WORD, dtype=torch.int32, device=DEV)
+        vote = torch.full((W + 4,), CANARY_WORD, dtype=torch.int32, device=DEV)
+        gd = torch.from_numpy(g).to(DEV)
+        if mode == "warmup":
+            B.signsgd_warmup_step(xd, gd, md, M, d, ld, beta, delta, bits, ldw, vote)
+            b_ref, v_ref = oracle.signsgd_warmup_step(x_ref, g.reshape(-1), m_ref, M, d, beta, delta, ld=ld, ldw=ldw)
+        else:
+            B.signsgd_step(xd, gd, md, M, d, ld, beta, delta, bits, ldw, vote)
+            b_ref, v_ref = oracle.signsgd_step(x_ref, g.reshape(-1), m_ref, M, d, beta, delta, ld=ld, ldw=ldw)
+        what = "seed=%d M=%d d=%d %s step %d" % (seed, M, d, mode, k)
+        check_rows(bits, b_ref, M, ldw, W, "bits " + what)
+        assert np.array_equal(u32(vote)[:W], v_ref), what
+        assert np.all(u32(vote)[W:] == np.uint32(0xDEADBEEF)), what
+        gx = f32(xd)
+        assert_same_f32(gx[:d], x_ref, "x " + what)
+        assert np.all(gx[d:] == np.float32(CANARY_F)), what
+        if with_m:
+            assert_same_f32(f32(md).reshape(-1), m_ref, "m " + what)
+
+
 # Odd vector lengths large enough that the launchers pick their largest tiles (16 and 32 elements per
 # thread: from about 64 Mi elements with a momentum, 32 Mi without), so that those instantiations meet a
 # ragged last tile, a last word with pad bits, and rows whose stride exceeds d.
