@@ -804,6 +804,33 @@ def test_vote_counts_and_sum_apply(M):
         assert np.all(gx[d:] == np.float32(CANARY_F))
 
 
+@pytest.mark.parametrize("seed", range(32))
+def test_vote_and_count_planes_random_shapes(seed):
+    """Seeded random worker counts (1 .. 1024, every kernel form: one row, 2 .. 7 rows, guarded and plain tails,
+    up to eleven planes), lengths and row strides; random words with garbage in the row padding; vote and count
+    planes against the oracle, canaries behind both outputs."""
+    r = np.random.default_rng(7000 + seed)
+    M = int(r.choice([1, 2, 3, 4, 5, 6, 7, 8, 9, 13, 16, 31, 32, 63, 64, 127, 128, 300, 1024])) if seed % 2 else int(r.integers(1, 130))
+    d = int(10 ** r.uniform(0.0, 5.3 if M <= 130 else 4.0))
+    W = oracle.words(d)
+    ldw, ldc = wl.round_up(W, 4) + 4 * int(r.integers(0, 3)), wl.round_up(W, 4) + 4 * int(r.integers(0, 3))
+    rows = r.integers(0, 2**32, size=(M, ldw), dtype=np.uint32)
+    rows[:, W - 1] &= np.uint32((1 << (d - 32 * (W - 1))) - 1 if d % 32 else 0xFFFFFFFF)   # pad bits 0, as the pack calls write them
+    bd = torch.from_numpy(rows.view(np.int32)).to(DEV)
+    vote = torch.full((W + 4,), CANARY_WORD, dtype=torch.int32, device=DEV)
+    B.majority_vote(bd, M, d, ldw, vote)
+    ref = oracle.majority_vote(rows.reshape(-1), M, d, ldw=ldw)
+    assert np.array_equal(u32(vote)[:W], ref), "vote seed=%d M=%d d=%d" % (seed, M, d)
+    assert np.all(u32(vote)[W:] == np.uint32(0xDEADBEEF))
+    NPc = M.bit_length()
+    counts = torch.full((NPc, ldc), CANARY_WORD, dtype=torch.int32, device=DEV)
+    B.vote_counts(bd, M, d, ldw, counts, ldc)
+    cref = oracle.vote_count_planes(rows.reshape(-1), M, d, ldw=ldw, ldc=ldc).reshape(NPc, ldc)
+    got = u32(counts)
+    assert np.array_equal(got[:, :W], cref[:, :W]), "counts seed=%d M=%d d=%d" % (seed, M, d)
+    assert np.all(got[:, W:] == np.uint32(0xDEADBEEF))
+
+
 # ------------------------------------------------------------------ majority vote with abstention
 
 @pytest.mark.parametrize("M", [1, 2, 3, 7, 8, 16, 33, 255, 1024])
