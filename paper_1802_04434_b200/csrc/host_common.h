@@ -124,6 +124,14 @@ inline bool vote_guarded(unsigned planes) {
   return planes >= (unsigned)kGuardedMinPlanes && planes <= (unsigned)kGuardedMaxPlanes;
 }
 
+// Vote of many rows on a short vector: the kernel that spreads the rows over the warps of a CTA (one CTA
+// per 32 chunks of four words), from 13 rows on, while its grid is at most 4 CTAs per SM (13 .. 23 rows:
+// d up to 2^21 on 148 SMs) or 8 CTAs per SM (24 rows and more: d up to 2^22); measured crossovers on B200.
+inline bool vote_split(size_t M, unsigned long long chunks, int sms) {
+  if (M < 13) return false;
+  return (chunks + 31) / 32 <= (M >= 24 ? 8ull : 4ull) * (unsigned long long)sms;
+}
+
 unsigned vote_planes(size_t M) {
   unsigned L = 0;
   while ((M / 2) >= (size_t(1) << L)) ++L;  // smallest L with floor(M/2) < 2^L

@@ -115,11 +115,13 @@ def test_majority_vote_small(M):
 
 @pytest.mark.parametrize("M,d", [(5, (1 << 25) + 37), (7, (1 << 25) + 37), (7, 5_000_003), (4, 3_000_001),
                                  (13, (1 << 24) + 4099), (31, 5_000_003), (63, 2_000_003), (64, 2_000_003),
-                                 (100, 1_000_003)])
+                                 (100, 1_000_003), (64, 5_000_003), (100, 5_000_003), (16, 3_000_001),
+                                 (16, 1_500_001)])
 def test_majority_vote_long_vectors(M, d):
     """The vote kernels (the one for exactly 2 .. 7 rows; the general one with its remaining rows as one guarded
-    batch, M = 8 .. 127, or in batches of 4, 2, 1) on launches many CTAs per SM deep and on shorter ones, with a
-    ragged last word and garbage in the row padding."""
+    batch, M = 8 .. 127, or in batches of 4, 2, 1; the one that spreads 13 and more rows over the warps of a CTA
+    while the vector is short: both sides of its threshold for M = 16, 64, 100) on launches many CTAs per SM deep
+    and on shorter ones, with a ragged last word and garbage in the row padding."""
     r = np.random.default_rng(M * 7919 + d % 1000)
     W = oracle.words(d)
     ldw = wl.round_up(W, 4) + 8
