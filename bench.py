@@ -43,15 +43,15 @@ FALLBACK_HBM_GBS = 6650.0
 # with the same M it is scaled (the path is elementwise, so traffic grows in proportion to d as long as
 # the operands exceed L2).  Valid only while the kernel sources are unchanged.
 NCU_TRAFFIC = {
-    "source_sha256": "59888e42af59cf931e8d6a962d2aade157fff204fbc5e3ea026383c3041b0187",
+    "source_sha256": "7257bc4e8464b4bc301ae59fd613c1dba7194e2a8919a9ec618576fd181ce183",
     "per_param": {
         # profiles/dram_bytes_worker_vote_apply_bertlarge_M16_full_size.md: a one-pass capture of the full-size
         # default workload (d = 335,141,888)
-        "worker_pack_kernel:M16": {"bytes_per_param": (42900220416 + 22068522496) / 335141888, "d": 335141888},
-        "vote_kernel:M16": {"bytes_per_param": (670310400 + 36460032) / 335141888, "d": 335141888},
-        "apply_kernel:M16": {"bytes_per_param": (1382524928 + 1277444352) / 335141888, "d": 335141888},
+        "worker_pack_kernel:M16": {"bytes_per_param": (42899410688 + 22068347136) / 335141888, "d": 335141888},
+        "vote_kernel:M16": {"bytes_per_param": (670312448 + 36816640) / 335141888, "d": 335141888},
+        "apply_kernel:M16": {"bytes_per_param": (1382548480 + 1277543680) / 335141888, "d": 335141888},
         # profiles/fused_step_kernel_resnet50_M7_ncu_full.md (captured at full size)
-        "fused_step_kernel:M7": {"bytes_per_param": (1.533714e9 + 795.096064e6) / 25557056, "d": 25557056},
+        "fused_step_kernel:M7": {"bytes_per_param": (1.533634e9 + 793.212160e6) / 25557056, "d": 25557056},
     },
 }
 
