@@ -1,5 +1,6 @@
-// Launchers of the direct (register-load) vote kernel, for the translation units that vote: the step
-// entry points and the count-plane variant.  Unnamed namespace: one copy per including unit.
+// Launchers of the direct (register-load) vote kernels (general, exact row count, rows split over warps), for the
+// translation units that vote: the step entry points and the count-plane variant.  Unnamed namespace: one copy per
+// including unit.
 #ifndef SSGD_VOTE_LAUNCH_H_
 #define SSGD_VOTE_LAUNCH_H_
 
